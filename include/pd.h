@@ -1,0 +1,148 @@
+/* pd.h - C ABI of the B200 (sm_100a) encoder-layer operator library.
+ *
+ * The operators are the ones the paper's search system exists to generate
+ * (Table "ML operators optimized using PerfLLM": softmax, layernorm, matmul,
+ * bmm, add), written in the loop-nest notation of Section 2.1
+ * "Representation" / Table "Supported representation features in PerfDojo",
+ * and chained into the forward pass of one post-LN transformer encoder layer.
+ *
+ * Conventions common to every entry point
+ *  - Pointers are DEVICE pointers unless a comment says "host".  The caller owns
+ *    every buffer (workspace included); the library allocates no device memory
+ *    and keeps no pointer after it returns.
+ *  - Tensors are dense and row-major.  Sizes are in elements, strides (ld*) too.
+ *  - Calls validate their arguments on the host, enqueue work on `stream` and
+ *    return without synchronising.  On any error nothing has been enqueued.
+ *  - A zero outer extent (rows == 0, M == 0, N == 0, batch == 0) is PD_OK and
+ *    launches nothing; a zero reduction extent (cols == 0, K == 0) is
+ *    PD_ERR_BAD_SHAPE.
+ *  - Results are deterministic: no atomics, fixed reduction trees.
+ *  - The current device must be compute capability 10.x, else PD_ERR_UNSUPPORTED.
+ *  - There is no CPU fallback of any kind.
+ */
+#ifndef PD_H_
+#define PD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef PD_NO_CUDA_HEADERS
+typedef struct CUstream_st* cudaStream_t;
+#else
+#include <cuda_runtime_api.h>
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  PD_OK = 0,
+  PD_ERR_NULL_POINTER = 1,
+  PD_ERR_BAD_SHAPE = 2,
+  PD_ERR_UNSUPPORTED = 3,
+  PD_ERR_ALIGNMENT = 4,
+  PD_ERR_WORKSPACE_TOO_SMALL = 5,
+  PD_ERR_CUDA = 6,
+  PD_ERR_DEVICE_TIMEOUT = 7
+} pd_status;
+
+typedef enum { PD_BF16 = 0, PD_F32 = 1 } pd_dtype;
+
+/* Human-readable name of a status; static storage, never null. */
+const char* pd_status_string(pd_status status);
+
+/* cudaError_t (as int) behind the calling thread's most recent PD_ERR_CUDA. */
+int pd_last_cuda_error(void);
+
+/* Every bounded wait inside the tensor-core kernels records a non-zero code in
+ * a device status word when it gives up (the kernel then drains and returns
+ * instead of hanging).  This call synchronises the current device, copies the
+ * word to *code (host pointer; 0 = no timeout since the last clear), and
+ * returns PD_ERR_DEVICE_TIMEOUT if it is non-zero.  pd_clear_device_status
+ * resets it. */
+pd_status pd_get_device_status(int* code);
+pd_status pd_clear_device_status(void);
+
+/* Row-wise softmax over the last dimension (operator "softmax" of the paper's
+ * operator table; reduction, broadcast and element-wise features):
+ *   y[i,j] = exp(x[i,j] - m_i) / sum_j exp(x[i,j] - m_i),  m_i = max_j x[i,j].
+ * x, y: fp32 [rows, cols], contiguous rows (ld == cols).  y may alias x.
+ * Fast paths need 16-byte aligned pointers and cols % 4 == 0; other shapes take
+ * a slower GPU path.  fp32 arithmetic, full-precision expf. */
+pd_status pd_softmax(const float* x, float* y, int64_t rows, int64_t cols, cudaStream_t stream);
+
+/* Layer normalisation over the last dimension (operators "layernorm 1/2"):
+ *   mu_i = mean_j x[i,j];  var_i = mean_j (x[i,j] - mu_i)^2   (biased, 1/cols)
+ *   y[i,j] = (x[i,j] - mu_i) / sqrt(var_i + eps) * gamma[j] + beta[j].
+ * x, y: fp32 [rows, cols]; gamma, beta: fp32 [cols].  y may alias x. */
+pd_status pd_layernorm(const float* x, const float* gamma, const float* beta, float* y,
+                       int64_t rows, int64_t cols, float eps, cudaStream_t stream);
+
+/* Fused bias + GELU(erf) + residual in one pass over HBM (element-wise and
+ * broadcast features; nearest paper operators "add" and "relu"):
+ *   out[i,j] = GELU(x[i,j] + bias[j]) + r[i,j],  GELU(z) = z/2 * (1 + erf(z/sqrt 2)).
+ * x, out: fp32 [rows, cols]; bias: fp32 [cols]; r: fp32 [rows, cols] or NULL
+ * (no residual term).  out may alias x or r. */
+pd_status pd_bias_gelu_residual(const float* x, const float* bias, const float* r, float* out,
+                                int64_t rows, int64_t cols, cudaStream_t stream);
+
+/* bf16 matrix product with fp32 accumulation on the tcgen05 tensor cores
+ * (operators "matmul" and, with batch > 1, "bmm"):
+ *   C[b][m,n] = sum_k A[b][m,k] * B[b][k,n].
+ * A: bf16 [M, K], row stride lda.  B: bf16, either [K, N] with row stride ldb
+ * (b_is_nk == 0) or stored transposed as [N, K] with row stride ldb
+ * (b_is_nk == 1).  C: [M, N], row stride ldc, bf16 (round-to-nearest-even) or
+ * fp32 per c_dtype.  Problem b starts strideA/strideB/strideC elements after
+ * problem b-1 (ignored when batch == 1).
+ * Requirements: 16-byte aligned base pointers; lda, ldb, strideA, strideB
+ * multiples of 8 elements; ldc * sizeof(C element) and strideC * sizeof(C
+ * element) multiples of 16 bytes (else PD_ERR_ALIGNMENT); ld* at least the
+ * row length; M, N, K otherwise arbitrary (ragged edges are zero-filled on load
+ * and clipped on store).  C must not overlap A or B. */
+pd_status pd_gemm_bf16(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K,
+                       int64_t lda, int64_t ldb, int64_t ldc, int b_is_nk, pd_dtype c_dtype,
+                       int64_t batch, int64_t strideA, int64_t strideB, int64_t strideC,
+                       cudaStream_t stream);
+
+/* Shape of one post-LN encoder layer (BERT-large: 32 x 512 tokens, hidden 1024,
+ * 16 heads of 64, FFN 4096).  hidden must equal heads * 64. */
+typedef struct {
+  int32_t batch, seq, hidden, heads, ffn;
+  float ln_eps;
+} pd_encoder_layer_desc;
+
+/* Weights of one layer.  Matrices are bf16 [in, out] row-major: w_qkv
+ * [hidden, 3*hidden] with column blocks [Q | K | V] and head h in columns
+ * 64h..64h+63 of each block; w_o [hidden, hidden]; w_ffn1 [hidden, ffn];
+ * w_ffn2 [ffn, hidden].  Biases and LayerNorm parameters are fp32 vectors. */
+typedef struct {
+  const void *w_qkv, *w_o, *w_ffn1, *w_ffn2;
+  const float *b_qkv, *b_o, *b_ffn1, *b_ffn2;
+  const float *ln1_gamma, *ln1_beta, *ln2_gamma, *ln2_beta;
+} pd_encoder_layer_weights;
+
+/* Bytes of caller-provided device workspace pd_encoder_layer_fwd needs for
+ * `desc` (0 if desc is NULL or invalid). */
+size_t pd_encoder_layer_workspace_bytes(const pd_encoder_layer_desc* desc);
+
+/* Forward pass of one encoder layer, no dropout, no mask, token t = b*seq + s:
+ *   QKV = X Wqkv + bqkv
+ *   Ctx[b,h] = softmax(Q[b,h] K[b,h]^T / sqrt(64)) V[b,h]
+ *   H1  = LayerNorm(Ctx Wo + bo + X; gamma1, beta1)
+ *   Mid = GELU(H1 W1 + b1)
+ *   Y   = LayerNorm(Mid W2 + b2 + H1; gamma2, beta2)
+ * desc, weights: host structs (device pointers inside).  x, y: bf16
+ * [batch*seq, hidden]; y must not overlap x or the workspace.  workspace: 256-
+ * byte aligned, at least pd_encoder_layer_workspace_bytes(desc) bytes, else
+ * PD_ERR_WORKSPACE_TOO_SMALL.  Contractions accumulate in fp32; softmax,
+ * LayerNorm statistics and the pre-LayerNorm sums are fp32; Q, K, V, the
+ * attention probabilities, Ctx, H1, Mid and Y are stored as bf16. */
+pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* weights,
+                               const void* x, void* y, void* workspace, size_t workspace_bytes,
+                               cudaStream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PD_H_ */

@@ -1,0 +1,94 @@
+// Status handling, device checks and the device status word of the pd library.
+#include "pd_common.cuh"
+
+namespace pd {
+namespace {
+
+thread_local int tl_last_cuda_error = 0;
+constexpr int kMaxDevices = 64;
+
+// Written by the bounded waits of the tensor-core kernels when they give up.
+__device__ int g_device_status;
+
+}  // namespace
+
+pd_status record_cuda_error(cudaError_t e) {
+  if (e == cudaSuccess) return PD_OK;
+  tl_last_cuda_error = (int)e;
+  return PD_ERR_CUDA;
+}
+
+pd_status require_sm100() {
+  static int cached_major[kMaxDevices];  // 0 = not queried yet
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  if (dev < 0 || dev >= kMaxDevices) return PD_ERR_UNSUPPORTED;
+  if (cached_major[dev] == 0) {
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    cached_major[dev] = major > 0 ? major : -1;
+  }
+  return cached_major[dev] == 10 ? PD_OK : PD_ERR_UNSUPPORTED;
+}
+
+int sm_count() {
+  static int cached[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
+  if (cached[dev] == 0) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+    cached[dev] = n;
+  }
+  return cached[dev];
+}
+
+int* device_status_ptr() {
+  static int* cached[kMaxDevices];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  if (!cached[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+    cached[dev] = static_cast<int*>(p);
+  }
+  return cached[dev];
+}
+
+}  // namespace pd
+
+extern "C" const char* pd_status_string(pd_status status) {
+  switch (status) {
+    case PD_OK: return "PD_OK";
+    case PD_ERR_NULL_POINTER: return "PD_ERR_NULL_POINTER";
+    case PD_ERR_BAD_SHAPE: return "PD_ERR_BAD_SHAPE";
+    case PD_ERR_UNSUPPORTED: return "PD_ERR_UNSUPPORTED";
+    case PD_ERR_ALIGNMENT: return "PD_ERR_ALIGNMENT";
+    case PD_ERR_WORKSPACE_TOO_SMALL: return "PD_ERR_WORKSPACE_TOO_SMALL";
+    case PD_ERR_CUDA: return "PD_ERR_CUDA";
+    case PD_ERR_DEVICE_TIMEOUT: return "PD_ERR_DEVICE_TIMEOUT";
+  }
+  return "PD_ERR_UNKNOWN";
+}
+
+extern "C" int pd_last_cuda_error(void) { return pd::tl_last_cuda_error; }
+
+extern "C" pd_status pd_get_device_status(int* code) {
+  if (!code) return PD_ERR_NULL_POINTER;
+  int* p = pd::device_status_ptr();
+  if (!p) return PD_ERR_CUDA;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemcpy(code, p, sizeof(int), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return pd::record_cuda_error(e);
+  return *code == 0 ? PD_OK : PD_ERR_DEVICE_TIMEOUT;
+}
+
+extern "C" pd_status pd_clear_device_status(void) {
+  int* p = pd::device_status_ptr();
+  if (!p) return PD_ERR_CUDA;
+  cudaError_t e = cudaDeviceSynchronize();
+  if (e == cudaSuccess) e = cudaMemset(p, 0, sizeof(int));
+  return pd::record_cuda_error(e);
+}

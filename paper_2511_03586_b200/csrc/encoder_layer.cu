@@ -1,0 +1,139 @@
+// Forward pass of one post-LN transformer encoder layer: a host-side driver that
+// chains the library's kernels on one stream with no host synchronisation.
+//
+//   QKV = X Wqkv + bqkv                                   (GEMM, bias epilogue)
+//   S   = Q K^T / 8, P = softmax(S), Ctx = P V  per head  (batched GEMM, softmax, batched GEMM)
+//   pre = Ctx Wo + bo + X                                 (GEMM, bias + residual epilogue, fp32)
+//   H1  = LayerNorm(pre)                                  (row kernel, bf16 out)
+//   Mid = GELU(H1 W1 + b1)                                (GEMM, bias + GELU epilogue)
+//   pre = Mid W2 + b2 + H1                                (GEMM, bias + residual epilogue, fp32)
+//   Y   = LayerNorm(pre)                                  (row kernel, bf16 out)
+#include "pd_common.cuh"
+
+namespace pd {
+namespace {
+
+constexpr int kHeadDim = 64;
+constexpr size_t kAlign = 256;
+
+inline size_t round_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct Workspace {
+  size_t qkv, scores, probs, ctx, pre, h1, mid, total;
+};
+
+bool valid_desc(const pd_encoder_layer_desc* d) {
+  if (!d) return false;
+  if (d->batch < 0 || d->seq <= 0 || d->hidden <= 0 || d->heads <= 0 || d->ffn <= 0) return false;
+  if (!(d->ln_eps >= 0.f)) return false;
+  return true;
+}
+
+bool supported_desc(const pd_encoder_layer_desc* d) {
+  return d->hidden == d->heads * kHeadDim && d->seq % 8 == 0 && d->ffn % 8 == 0;
+}
+
+Workspace plan(const pd_encoder_layer_desc* d) {
+  const size_t T = (size_t)d->batch * d->seq, H = d->hidden, F = d->ffn, S = d->seq;
+  const size_t score_elems = (size_t)d->batch * d->heads * S * S;
+  Workspace w{};
+  size_t off = 0;
+  w.qkv = off; off += round_up(T * 3 * H * 2);
+  w.scores = off; off += round_up(score_elems * 4);
+  w.probs = off; off += round_up(score_elems * 2);
+  w.ctx = off; off += round_up(T * H * 2);
+  w.pre = off; off += round_up(T * H * 4);
+  w.h1 = off; off += round_up(T * H * 2);
+  w.mid = off; off += round_up(T * F * 2);
+  w.total = off;
+  return w;
+}
+
+}  // namespace
+}  // namespace pd
+
+extern "C" size_t pd_encoder_layer_workspace_bytes(const pd_encoder_layer_desc* desc) {
+  if (!pd::valid_desc(desc) || !pd::supported_desc(desc)) return 0;
+  return pd::plan(desc).total;
+}
+
+extern "C" pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* w,
+                                          const void* x, void* y, void* workspace, size_t workspace_bytes,
+                                          cudaStream_t stream) {
+  using namespace pd;
+  if (!desc || !w || !x || !y) return PD_ERR_NULL_POINTER;
+  if (!w->w_qkv || !w->w_o || !w->w_ffn1 || !w->w_ffn2 || !w->b_qkv || !w->b_o || !w->b_ffn1 || !w->b_ffn2 ||
+      !w->ln1_gamma || !w->ln1_beta || !w->ln2_gamma || !w->ln2_beta)
+    return PD_ERR_NULL_POINTER;
+  if (!valid_desc(desc)) return PD_ERR_BAD_SHAPE;
+  if (!supported_desc(desc)) return PD_ERR_UNSUPPORTED;
+  const void* ptrs[] = {x, y, w->w_qkv, w->w_o, w->w_ffn1, w->w_ffn2, w->b_qkv, w->b_o, w->b_ffn1, w->b_ffn2,
+                        w->ln1_gamma, w->ln1_beta, w->ln2_gamma, w->ln2_beta};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return PD_ERR_ALIGNMENT;
+  if (desc->batch == 0) return PD_OK;
+  const Workspace ws = plan(desc);
+  if (!workspace) return PD_ERR_NULL_POINTER;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return PD_ERR_ALIGNMENT;
+  if (workspace_bytes < ws.total) return PD_ERR_WORKSPACE_TOO_SMALL;
+  pd_status st = require_sm100();
+  if (st != PD_OK) return st;
+
+  const int64_t B = desc->batch, S = desc->seq, H = desc->hidden, NH = desc->heads, F = desc->ffn, T = B * S;
+  uint8_t* base = static_cast<uint8_t*>(workspace);
+  auto* qkv = reinterpret_cast<__nv_bfloat16*>(base + ws.qkv);
+  auto* scores = reinterpret_cast<float*>(base + ws.scores);
+  auto* probs = reinterpret_cast<__nv_bfloat16*>(base + ws.probs);
+  auto* ctx = reinterpret_cast<__nv_bfloat16*>(base + ws.ctx);
+  auto* pre = reinterpret_cast<float*>(base + ws.pre);
+  auto* h1 = reinterpret_cast<__nv_bfloat16*>(base + ws.h1);
+  auto* mid = reinterpret_cast<__nv_bfloat16*>(base + ws.mid);
+  const auto* xb = static_cast<const __nv_bfloat16*>(x);
+
+  {  // QKV projection
+    GemmProblem g;
+    g.A = x; g.B = w->w_qkv; g.C = qkv; g.M = T; g.N = 3 * H; g.K = H; g.lda = H; g.ldb = 3 * H; g.ldc = 3 * H;
+    g.bias = w->b_qkv;
+    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+  }
+  {  // scores = Q K^T / sqrt(64), fp32, one [S, S] block per (batch, head)
+    GemmProblem g;
+    g.A = qkv; g.B = qkv + H; g.C = scores; g.M = S; g.N = S; g.K = kHeadDim; g.lda = 3 * H; g.ldb = 3 * H; g.ldc = S;
+    g.b_is_nk = true; g.c_dtype = PD_F32; g.alpha = 0.125f;
+    g.batch_inner = NH; g.batch_outer = B;
+    g.strideA_inner = kHeadDim; g.strideA_outer = S * 3 * H;
+    g.strideB_inner = kHeadDim; g.strideB_outer = S * 3 * H;
+    g.strideC_inner = S * S; g.strideC_outer = NH * S * S;
+    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+  }
+  if ((st = launch_softmax(scores, probs, true, B * NH * S, S, stream)) != PD_OK) return st;
+  {  // Ctx = P V, heads written back to their column blocks
+    GemmProblem g;
+    g.A = probs; g.B = qkv + 2 * H; g.C = ctx; g.M = S; g.N = kHeadDim; g.K = S; g.lda = S; g.ldb = 3 * H; g.ldc = H;
+    g.batch_inner = NH; g.batch_outer = B;
+    g.strideA_inner = S * S; g.strideA_outer = NH * S * S;
+    g.strideB_inner = kHeadDim; g.strideB_outer = S * 3 * H;
+    g.strideC_inner = kHeadDim; g.strideC_outer = S * H;
+    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+  }
+  {  // output projection + bias + residual (fp32 sum kept for the LayerNorm)
+    GemmProblem g;
+    g.A = ctx; g.B = w->w_o; g.C = pre; g.M = T; g.N = H; g.K = H; g.lda = H; g.ldb = H; g.ldc = H;
+    g.c_dtype = PD_F32; g.bias = w->b_o; g.residual = xb; g.ldr = H;
+    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+  }
+  if ((st = launch_layernorm(pre, w->ln1_gamma, w->ln1_beta, h1, true, T, H, desc->ln_eps, stream)) != PD_OK) return st;
+  {  // FFN up + bias + GELU
+    GemmProblem g;
+    g.A = h1; g.B = w->w_ffn1; g.C = mid; g.M = T; g.N = F; g.K = H; g.lda = H; g.ldb = F; g.ldc = F;
+    g.bias = w->b_ffn1; g.gelu = true;
+    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+  }
+  {  // FFN down + bias + residual
+    GemmProblem g;
+    g.A = mid; g.B = w->w_ffn2; g.C = pre; g.M = T; g.N = H; g.K = F; g.lda = F; g.ldb = H; g.ldc = H;
+    g.c_dtype = PD_F32; g.bias = w->b_ffn2; g.residual = h1; g.ldr = H;
+    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+  }
+  return launch_layernorm(pre, w->ln2_gamma, w->ln2_beta, y, true, T, H, desc->ln_eps, stream);
+}

@@ -1,0 +1,436 @@
+// bf16 x bf16 -> fp32 contraction on the tcgen05 tensor cores with a fused epilogue.
+//
+//   C[m,n] = act(alpha * sum_k A[m,k] B[k,n] + bias[n]) + residual[m,n]
+//
+// Persistent, warp-specialised kernel, one CTA of 192 threads per SM:
+//   warp 0, one lane : TMA producer.  Streams 128 x 64 tiles of A and BN x 64
+//                      tiles of B (128-byte swizzle) into a ring of shared-memory
+//                      stages; a "full" mbarrier per stage counts the bytes.
+//   warp 1, one lane : MMA issuer.  Four tcgen05.mma (128 x BN x 16) per stage
+//                      accumulate into one of two TMEM accumulators; a
+//                      tcgen05.commit hands the stage back ("empty" barrier) and,
+//                      after the last k-block, publishes the accumulator.
+//   warps 2-5        : epilogue.  Each warp drains its 32 TMEM lanes (32 rows of
+//                      the tile) 32 columns at a time, applies the epilogue in
+//                      fp32 and writes C, while the MMA warp already fills the
+//                      other accumulator with the next tile.
+// B is taken either as [K, N] (N contiguous: an "MN-major" MMA operand, loaded
+// as BN/64 boxes of 64 x 64) or as [N, K] (K contiguous, "K-major").  Ragged M,
+// N, K edges are zero-filled by TMA on load and predicated on store.
+// Every mbarrier wait is bounded: on expiry the kernel records a code in the
+// device status word, all roles drain, tensor memory is freed and the kernel
+// returns.
+#include "pd_common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace pd {
+namespace {
+
+using namespace sm100;
+
+constexpr int BM = 128;       // tile rows = TMEM lanes
+constexpr int BK = 64;        // k-block: 64 bf16 = one 128-byte swizzle row
+constexpr int UMMA_K = 16;    // k extent of one tcgen05.mma for 16-bit inputs
+constexpr int kThreads = 192;
+constexpr int kEpilogueThreads = 128;
+constexpr int kSmemLimit = 227 * 1024;
+
+template <int BN>
+struct Cfg {
+  static constexpr int kStageA = BM * BK * 2;
+  static constexpr int kStageB = BN * BK * 2;
+  static constexpr int kStage = kStageA + kStageB;
+  static constexpr int kBarrierBytes = 1024;
+  static constexpr int kStagesMax = (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes) / kStage;
+  static constexpr int kStages = kStagesMax > 8 ? 8 : kStagesMax;
+  static constexpr int kSmemBytes = kStages * kStage + kBarrierBytes + 1024;
+  static constexpr int kTmemCols = 2 * BN;  // two accumulators; 128, 256 or 512: a power of two
+};
+
+struct KernelParams {
+  void* C;
+  const float* bias;
+  const __nv_bfloat16* residual;
+  int* status;
+  int64_t ldc, strideC_inner, strideC_outer, ldr;
+  int M, N, K;
+  int tiles_m, tiles_n, batch_inner, num_tiles;  // num_tiles = batch_outer * batch_inner * tiles_m * tiles_n
+  float alpha;
+  int c_is_f32, gelu;
+};
+
+// Codes left in the device status word by an expired wait.
+enum : int { kTimeoutProducer = 101, kTimeoutMmaFull = 102, kTimeoutMmaAcc = 103, kTimeoutEpilogue = 104 };
+
+__device__ __forceinline__ float gelu_erf(float z) {
+  return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int BN, bool B_NK>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                         const KernelParams p) {
+  using C = Cfg<BN>;
+  constexpr int kStages = C::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  // 128-byte swizzled tiles must start on a 1024-byte boundary.
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar_base = smem_base + kStages * C::kStage;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
+  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * kStages + 4);
+  uint8_t* ctrl = smem_gen + kStages * C::kStage + 8 * (2 * kStages + 5);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = (p.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(acc_full_bar(a), 1);
+      mbar_init(acc_empty_bar(a), kEpilogueThreads);
+    }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), C::kTmemCols);
+    tmem_relinquish_alloc_permit();
+  }
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      prefetch_tensormap(&tmap_a);
+      prefetch_tensormap(&tmap_b);
+      uint32_t it = 0;  // k-blocks issued so far, over all tiles
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+        const int nt = tile % p.tiles_n;
+        const int mt = (tile / p.tiles_n) % p.tiles_m;
+        const int b = tile / (p.tiles_n * p.tiles_m);
+        const int bi = b % p.batch_inner, bo = b / p.batch_inner;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
+          const uint32_t sa = smem_base + s * C::kStage, sb = sa + C::kStageA;
+          mbar_arrive_expect_tx(full_bar(s), C::kStage);
+          tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, bi, bo);
+          if (B_NK) {
+            tma_load_4d(sb, &tmap_b, full_bar(s), kb * BK, nt * BN, bi, bo);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j)
+              tma_load_4d(sb + j * (64 * BK * 2), &tmap_b, full_bar(s), nt * BN + j * 64, kb * BK, bi, bo);
+          }
+        }
+      }
+      if (!ok) {
+        // Leave no copy in flight: wait (briefly) for every stage last armed.
+        const uint32_t issued = it;
+        for (int s = 0; s < kStages; ++s) {
+          if ((uint32_t)s >= issued) break;
+          const uint32_t last = ((issued - 1 - s) / kStages) * kStages + s;
+          volatile int never = 0;
+          int sink = 0;
+          mbar_wait(full_bar(s), (last / kStages) & 1u, &never, &sink, 0, 20000000ull);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // --------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(BM, BN, false, !B_NK);
+      uint32_t it = 0;
+      int local = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local) {
+        const int acc = local & 1;
+        const uint32_t acc_ph = (local >> 1) & 1u;
+        if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc)) { ok = false; break; }
+        tcgen05_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
+          tcgen05_fence_after_sync();
+          const uint32_t sa = smem_base + s * C::kStage, sb = sa + C::kStageA;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
+            const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
+                                         : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
+            mma_bf16_ss(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma_commit(empty_bar(s));
+        }
+        if (ok) mma_commit(acc_full_bar(acc));
+      }
+      if (!ok) {
+        // Let every MMA already issued finish before tensor memory is freed.
+        mma_commit(drain_bar);
+        volatile int never = 0;
+        int sink = 0;
+        mbar_wait(drain_bar, 0, &never, &sink, 0, 20000000ull);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;  // TMEM lanes 32*quarter .. 32*quarter+31 belong to this warp
+    const int row_in_tile = quarter * 32 + lane;
+    int local = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local) {
+      const int nt = tile % p.tiles_n;
+      const int mt = (tile / p.tiles_n) % p.tiles_m;
+      const int b = tile / (p.tiles_n * p.tiles_m);
+      const int bi = b % p.batch_inner, bo = b / p.batch_inner;
+      const int acc = local & 1;
+      const uint32_t acc_ph = (local >> 1) & 1u;
+      if (!mbar_wait(acc_full_bar(acc), acc_ph, abort_flag, p.status, kTimeoutEpilogue)) { ok = false; break; }
+      tcgen05_fence_after_sync();
+      const int m = mt * BM + row_in_tile;
+      const bool row_ok = m < p.M;
+      const int64_t c_row = (int64_t)bo * p.strideC_outer + (int64_t)bi * p.strideC_inner + (int64_t)m * p.ldc;
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        const int n0 = nt * BN + c0;
+        if (n0 >= p.N) break;  // uniform over the warp
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(t_row + c0, r);
+        tmem_ld_wait();
+        if (!row_ok) continue;
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * p.alpha;
+        const bool full = n0 + 32 <= p.N;
+        if (p.bias) {
+          if (full) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+              const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias + n0 + j));
+              v[j] += bv.x; v[j + 1] += bv.y; v[j + 2] += bv.z; v[j + 3] += bv.w;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n0 + j < p.N) v[j] += __ldg(p.bias + n0 + j);
+          }
+        }
+        if (p.gelu) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+        }
+        if (p.residual) {
+          const __nv_bfloat16* rr = p.residual + (int64_t)m * p.ldr + n0;
+          if (full) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              const uint4 u = __ldg(reinterpret_cast<const uint4*>(rr + j));
+              const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+              for (int t = 0; t < 4; ++t) {
+                v[j + 2 * t] += __uint_as_float(w[t] << 16);
+                v[j + 2 * t + 1] += __uint_as_float(w[t] & 0xffff0000u);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n0 + j < p.N) v[j] += __bfloat162float(rr[j]);
+          }
+        }
+        if (p.c_is_f32) {
+          float* out = static_cast<float*>(p.C) + c_row + n0;
+          if (full) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(out + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n0 + j < p.N) out[j] = v[j];
+          }
+        } else {
+          __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.C) + c_row + n0;
+          if (full) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              uint4 u;
+              u.x = pack_bf16(v[j], v[j + 1]);
+              u.y = pack_bf16(v[j + 2], v[j + 3]);
+              u.z = pack_bf16(v[j + 4], v[j + 5]);
+              u.w = pack_bf16(v[j + 6], v[j + 7]);
+              *reinterpret_cast<uint4*>(out + j) = u;
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (n0 + j < p.N) out[j] = __float2bfloat16_rn(v[j]);
+          }
+        }
+      }
+      tcgen05_fence_before_sync();
+      mbar_arrive(acc_empty_bar(acc));
+    }
+  }
+
+  // ------------------------------------------------------------------- teardown
+  __syncwarp();
+  tcgen05_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tcgen05_fence_after_sync();
+    tmem_dealloc(tmem_base, C::kTmemCols);
+  }
+}
+
+// ---- host side -----------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+// bf16 tensor [outer][inner][rows][cols] with cols contiguous, 128-byte swizzle,
+// zero fill outside the extents.  Strides in elements.
+bool make_bf16_map(CUtensorMap* map, const void* base, int64_t cols, int64_t rows, int64_t ld, int64_t n_inner,
+                   int64_t stride_inner, int64_t n_outer, int64_t stride_outer, int box_cols, int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  // Unit batch extents still need a legal (16-byte multiple) stride.
+  if (n_inner == 1) stride_inner = ld * rows;
+  if (n_outer == 1) stride_outer = (n_inner == 1 ? ld * rows : stride_inner * n_inner);
+  const cuuint64_t dims[4] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)n_inner, (cuuint64_t)n_outer};
+  const cuuint64_t strides[3] = {(cuuint64_t)ld * 2, (cuuint64_t)stride_inner * 2, (cuuint64_t)stride_outer * 2};
+  const cuuint32_t box[4] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, bool B_NK>
+pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
+  using C = Cfg<BN>;
+  CUtensorMap ta, tb;
+  if (!make_bf16_map(&ta, g.A, g.K, g.M, g.lda, g.batch_inner, g.strideA_inner, g.batch_outer, g.strideA_outer, BK, BM))
+    return PD_ERR_UNSUPPORTED;
+  const bool okb = B_NK ? make_bf16_map(&tb, g.B, g.K, g.N, g.ldb, g.batch_inner, g.strideB_inner, g.batch_outer,
+                                        g.strideB_outer, BK, BN)
+                        : make_bf16_map(&tb, g.B, g.N, g.K, g.ldb, g.batch_inner, g.strideB_inner, g.batch_outer,
+                                        g.strideB_outer, 64, BK);
+  if (!okb) return PD_ERR_UNSUPPORTED;
+
+  KernelParams p{};
+  p.C = g.C; p.bias = g.bias; p.residual = g.residual; p.status = device_status_ptr();
+  if (!p.status) return PD_ERR_CUDA;
+  p.ldc = g.ldc; p.strideC_inner = g.strideC_inner; p.strideC_outer = g.strideC_outer; p.ldr = g.ldr;
+  p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
+  p.tiles_m = (int)((g.M + BM - 1) / BM);
+  p.tiles_n = (int)((g.N + BN - 1) / BN);
+  p.batch_inner = (int)g.batch_inner;
+  const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n * g.batch_inner * g.batch_outer;
+  if (tiles > 0x7fffffff) return PD_ERR_BAD_SHAPE;
+  p.num_tiles = (int)tiles;
+  p.alpha = g.alpha; p.c_is_f32 = g.c_dtype == PD_F32; p.gelu = g.gelu;
+
+  auto kernel = gemm_bf16_tcgen05_kernel<BN, B_NK>;
+  static bool attr_set = false;  // per template instantiation
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    attr_set = true;
+  }
+  const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
+  kernel<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, p);
+  return check_launch();
+}
+
+}  // namespace
+
+pd_status launch_gemm(const GemmProblem& g, cudaStream_t s) {
+  // 128 x 256 tiles have the best operand reuse; narrower tiles are used when N
+  // is small or when they fill the last wave of SMs noticeably better.
+  const int sms = sm_count();
+  auto waves_cost = [&](int bn) {
+    const int64_t tiles = ((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn) * g.batch_inner * g.batch_outer;
+    const int64_t waves = (tiles + sms - 1) / sms;
+    return (double)waves * bn;  // time ~ waves x tile width
+  };
+  int bn = 256;
+  if (g.N <= 64) bn = 64;
+  else if (g.N <= 128) bn = 128;
+  else if (waves_cost(128) * 1.08 < waves_cost(256)) bn = 128;
+  if (g.b_is_nk) {
+    if (bn == 256) return launch_variant<256, true>(g, s);
+    if (bn == 128) return launch_variant<128, true>(g, s);
+    return launch_variant<64, true>(g, s);
+  }
+  if (bn == 256) return launch_variant<256, false>(g, s);
+  if (bn == 128) return launch_variant<128, false>(g, s);
+  return launch_variant<64, false>(g, s);
+}
+
+}  // namespace pd
+
+extern "C" pd_status pd_gemm_bf16(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K,
+                                  int64_t lda, int64_t ldb, int64_t ldc, int b_is_nk, pd_dtype c_dtype,
+                                  int64_t batch, int64_t strideA, int64_t strideB, int64_t strideC,
+                                  cudaStream_t stream) {
+  if (!A || !B || !C) return PD_ERR_NULL_POINTER;
+  if (M < 0 || N < 0 || K <= 0 || batch < 0) return PD_ERR_BAD_SHAPE;
+  if (c_dtype != PD_BF16 && c_dtype != PD_F32) return PD_ERR_BAD_SHAPE;
+  if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff || batch > 0x7fffffff) return PD_ERR_BAD_SHAPE;
+  const int64_t b_cols = b_is_nk ? K : N;
+  if (lda < K || ldb < b_cols || ldc < N) return PD_ERR_BAD_SHAPE;
+  const int64_t c_elems_per_16B = c_dtype == PD_F32 ? 4 : 8;
+  if (!pd::aligned16(A) || !pd::aligned16(B) || !pd::aligned16(C) || lda % 8 || ldb % 8 || ldc % c_elems_per_16B)
+    return PD_ERR_ALIGNMENT;
+  if (batch > 1) {
+    if (strideA < 0 || strideB < 0 || strideC < 0) return PD_ERR_BAD_SHAPE;
+    if (strideA % 8 || strideB % 8 || strideC % c_elems_per_16B) return PD_ERR_ALIGNMENT;
+    if (strideA == 0 || strideB == 0) return PD_ERR_UNSUPPORTED;  // broadcast operands: not supported
+  }
+  if (M == 0 || N == 0 || batch == 0) return PD_OK;
+  pd_status st = pd::require_sm100();
+  if (st != PD_OK) return st;
+  pd::GemmProblem g;
+  g.A = A; g.B = B; g.C = C; g.M = M; g.N = N; g.K = K; g.lda = lda; g.ldb = ldb; g.ldc = ldc;
+  g.b_is_nk = b_is_nk != 0; g.c_dtype = c_dtype;
+  g.batch_inner = batch; g.batch_outer = 1;
+  g.strideA_inner = strideA; g.strideB_inner = strideB; g.strideC_inner = strideC;
+  return pd::launch_gemm(g, stream);
+}

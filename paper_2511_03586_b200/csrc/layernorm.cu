@@ -1,0 +1,190 @@
+// Layer normalisation over the last dimension, fp32 in, fp32 or bf16 out.
+//
+//   mu_i = mean_j x[i,j];  var_i = mean_j (x[i,j] - mu_i)^2  (biased)
+//   y[i,j] = (x[i,j] - mu_i) * rsqrt(var_i + eps) * gamma[j] + beta[j]
+//
+// HBM-bound: 8 bytes per element.  The row is read once into registers with
+// 128-bit loads; the mean and the centred second moment are then passes over
+// registers (data centred before squaring, mean refined by the mean of the
+// residuals: no E[x^2] - mu^2 cancellation), reduced with warp shuffles.
+//   * cols <= 1024   : one warp per row
+//   * cols <= 16384  : one CTA of 512 threads per row
+//   * otherwise      : one CTA per row, three passes from global/L2; partial
+//                      statistics are merged pairwise (Chan/Welford form)
+#include "pd_common.cuh"
+
+namespace pd {
+namespace {
+
+template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA, typename OutT>
+__global__ void __launch_bounds__(THREADS_PER_CTA)
+layernorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__ gamma,
+                            const float* __restrict__ beta, OutT* __restrict__ y, int64_t rows, int cols,
+                            float eps) {
+  constexpr int ROWS_PER_CTA = THREADS_PER_CTA / THREADS_PER_ROW;
+  constexpr int NWARPS = THREADS_PER_ROW / 32;
+  __shared__ float scratch[3][NWARPS];
+  const int t = threadIdx.x % THREADS_PER_ROW;
+  const int cols4 = cols >> 2;
+  const float inv_cols = 1.0f / (float)cols;
+  const float4* g4 = reinterpret_cast<const float4*>(gamma);
+  const float4* b4 = reinterpret_cast<const float4*>(beta);
+  for (int64_t row = (int64_t)blockIdx.x * ROWS_PER_CTA + threadIdx.x / THREADS_PER_ROW; row < rows;
+       row += (int64_t)gridDim.x * ROWS_PER_CTA) {
+    const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
+    float4 v[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int c = t + i * THREADS_PER_ROW;
+      v[i] = (c < cols4) ? ld_stream(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+    const float mu0 = block_reduce<NWARPS, false>(s, scratch, 0) * inv_cols;
+    // Centre on the first estimate, then refine it with the mean of the
+    // residuals: the fp32 sum above loses digits when |mean| >> spread, the sum
+    // of the (small) residuals does not.
+    float d1 = 0.f, d2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int c = t + i * THREADS_PER_ROW;
+      if (c < cols4) {
+        v[i].x -= mu0; v[i].y -= mu0; v[i].z -= mu0; v[i].w -= mu0;
+        d1 += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+        d2 += (v[i].x * v[i].x + v[i].y * v[i].y) + (v[i].z * v[i].z + v[i].w * v[i].w);
+      }
+    }
+    const float delta = block_reduce<NWARPS, false>(d1, scratch, 1) * inv_cols;
+    const float var = fmaxf(block_reduce<NWARPS, false>(d2, scratch, 2) * inv_cols - delta * delta, 0.f);
+    const float rstd = rsqrtf(var + eps);
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int c = t + i * THREADS_PER_ROW;
+      if (c < cols4) {
+        const float4 g = __ldg(g4 + c), b = __ldg(b4 + c);
+        store_out4(y, row * cols4 + c,
+                   make_float4((v[i].x - delta) * rstd * g.x + b.x, (v[i].y - delta) * rstd * g.y + b.y,
+                               (v[i].z - delta) * rstd * g.z + b.z, (v[i].w - delta) * rstd * g.w + b.w));
+      }
+    }
+    if constexpr (NWARPS > 1) __syncthreads();
+  }
+}
+
+// (count, mean, M2) partial statistics and their pairwise merge.
+struct Moments {
+  float n, mean, m2;
+};
+__device__ __forceinline__ Moments merge(Moments a, Moments b) {
+  const float n = a.n + b.n;
+  if (n == 0.f) return a;
+  const float d = b.mean - a.mean, w = b.n / n;
+  return Moments{n, a.mean + d * w, a.m2 + b.m2 + d * d * a.n * w};
+}
+
+template <typename OutT>
+__global__ void __launch_bounds__(256)
+layernorm_rows_generic(const float* __restrict__ x, const float* __restrict__ gamma,
+                       const float* __restrict__ beta, OutT* __restrict__ y, int64_t rows, int64_t cols,
+                       float eps) {
+  __shared__ Moments part[8];
+  __shared__ float stat[2];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+    const float* xr = x + row * cols;
+    // per-thread Welford over a strided slice of the row
+    Moments m{0.f, 0.f, 0.f};
+    for (int64_t j = threadIdx.x; j < cols; j += 256) {
+      const float v = xr[j];
+      m.n += 1.f;
+      const float d = v - m.mean;
+      m.mean += d / m.n;
+      m.m2 += d * (v - m.mean);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      Moments other{__shfl_xor_sync(0xffffffffu, m.n, o), __shfl_xor_sync(0xffffffffu, m.mean, o),
+                    __shfl_xor_sync(0xffffffffu, m.m2, o)};
+      // merge in a lane-independent order so that every lane ends with the same bits
+      m = (lane & o) ? merge(other, m) : merge(m, other);
+    }
+    if (lane == 0) part[warp] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      Moments tot = part[0];
+      for (int w = 1; w < 8; ++w) tot = merge(tot, part[w]);
+      stat[0] = tot.mean;
+      stat[1] = rsqrtf(tot.m2 / (float)cols + eps);
+    }
+    __syncthreads();
+    const float mu = stat[0], rstd = stat[1];
+    for (int64_t j = threadIdx.x; j < cols; j += 256)
+      store_out1(y, row * cols + j, (xr[j] - mu) * rstd * gamma[j] + beta[j]);
+    __syncthreads();
+  }
+}
+
+template <int VPT, typename OutT>
+void launch_warp_rows(const float* x, const float* g, const float* b, OutT* y, int64_t rows, int cols, float eps,
+                      cudaStream_t s) {
+  constexpr int kThreads = 256, kRowsPerCta = kThreads / 32;
+  const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
+  const int grid = (int)(ctas < (int64_t)sm_count() * 64 ? ctas : (int64_t)sm_count() * 64);
+  layernorm_rows_in_registers<VPT, 32, kThreads, OutT><<<grid, kThreads, 0, s>>>(x, g, b, y, rows, cols, eps);
+}
+
+template <int VPT, typename OutT>
+void launch_cta_rows(const float* x, const float* g, const float* b, OutT* y, int64_t rows, int cols, float eps,
+                     cudaStream_t s) {
+  constexpr int kThreads = 512;
+  const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
+  layernorm_rows_in_registers<VPT, kThreads, kThreads, OutT><<<grid, kThreads, 0, s>>>(x, g, b, y, rows, cols, eps);
+}
+
+template <typename OutT>
+pd_status dispatch(const float* x, const float* g, const float* b, OutT* y, int64_t rows, int64_t cols, float eps,
+                   cudaStream_t s) {
+  const bool vec_ok = (cols % 4 == 0) && aligned16(x) && aligned16(g) && aligned16(b) &&
+                      ((reinterpret_cast<uintptr_t>(y) & (sizeof(OutT) * 4 - 1)) == 0);
+  if (vec_ok && cols <= 1024) {
+    const int c = (int)cols;
+    if (c <= 128) launch_warp_rows<1>(x, g, b, y, rows, c, eps, s);
+    else if (c <= 256) launch_warp_rows<2>(x, g, b, y, rows, c, eps, s);
+    else if (c <= 512) launch_warp_rows<4>(x, g, b, y, rows, c, eps, s);
+    else launch_warp_rows<8>(x, g, b, y, rows, c, eps, s);
+  } else if (vec_ok && cols <= 16384) {
+    const int c = (int)cols;
+    if (c <= 2048) launch_cta_rows<1>(x, g, b, y, rows, c, eps, s);
+    else if (c <= 4096) launch_cta_rows<2>(x, g, b, y, rows, c, eps, s);
+    else if (c <= 8192) launch_cta_rows<4>(x, g, b, y, rows, c, eps, s);
+    else launch_cta_rows<8>(x, g, b, y, rows, c, eps, s);
+  } else {
+    const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
+    layernorm_rows_generic<OutT><<<grid, 256, 0, s>>>(x, g, b, y, rows, cols, eps);
+  }
+  return check_launch();
+}
+
+}  // namespace
+
+pd_status launch_layernorm(const float* x, const float* gamma, const float* beta, void* y, bool y_is_bf16,
+                           int64_t rows, int64_t cols, float eps, cudaStream_t s) {
+  if (y_is_bf16) return dispatch(x, gamma, beta, static_cast<__nv_bfloat16*>(y), rows, cols, eps, s);
+  return dispatch(x, gamma, beta, static_cast<float*>(y), rows, cols, eps, s);
+}
+
+}  // namespace pd
+
+extern "C" pd_status pd_layernorm(const float* x, const float* gamma, const float* beta, float* y, int64_t rows,
+                                  int64_t cols, float eps, cudaStream_t stream) {
+  if (!x || !gamma || !beta || !y) return PD_ERR_NULL_POINTER;
+  if (rows < 0 || cols <= 0 || !(eps >= 0.f)) return PD_ERR_BAD_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(gamma) |
+       reinterpret_cast<uintptr_t>(beta)) & 3u)
+    return PD_ERR_ALIGNMENT;
+  if (rows == 0) return PD_OK;
+  pd_status st = pd::require_sm100();
+  if (st != PD_OK) return st;
+  return pd::launch_layernorm(x, gamma, beta, y, false, rows, cols, eps, stream);
+}

@@ -1,0 +1,109 @@
+// Shared host/device helpers of the pd library (internal; not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pd.h"
+
+namespace pd {
+
+constexpr int kWarp = 32;
+
+// ---- host side -----------------------------------------------------------
+// Records `e` for pd_last_cuda_error() and maps it to a status.
+pd_status record_cuda_error(cudaError_t e);
+// cudaGetLastError() after a launch, mapped to a status.
+inline pd_status check_launch() { return record_cuda_error(cudaGetLastError()); }
+// PD_OK when the current device is compute capability 10.x.
+pd_status require_sm100();
+// Number of SMs of the current device (cached per device).
+int sm_count();
+// Device address of the status word the bounded waits report to (nullptr on failure).
+int* device_status_ptr();
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ---- device side ---------------------------------------------------------
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Block-wide reductions over NWARPS warps through a small shared array; every
+// thread receives the result.  `slot` selects one of two scratch rows so that
+// back-to-back reductions need only one barrier each.
+template <int NWARPS, bool IS_MAX>
+__device__ __forceinline__ float block_reduce(float v, float (*scratch)[NWARPS], int slot) {
+  v = IS_MAX ? warp_max(v) : warp_sum(v);
+  if constexpr (NWARPS == 1) return v;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane == 0) scratch[slot][warp] = v;
+  __syncthreads();
+  float r = scratch[slot][0];
+#pragma unroll
+  for (int w = 1; w < NWARPS; ++w) r = IS_MAX ? fmaxf(r, scratch[slot][w]) : r + scratch[slot][w];
+  return r;
+}
+
+// Streaming 128-bit global accesses: inputs are read once and outputs written
+// once, so neither should displace reusable lines.
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
+
+__device__ __forceinline__ void store_out4(float* base, int64_t idx4, float4 v) {
+  st_stream(reinterpret_cast<float4*>(base) + idx4, v);
+}
+__device__ __forceinline__ void store_out4(__nv_bfloat16* base, int64_t idx4, float4 v) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u;
+  u.x = *reinterpret_cast<uint32_t*>(&lo);
+  u.y = *reinterpret_cast<uint32_t*>(&hi);
+  __stcs(reinterpret_cast<uint2*>(base) + idx4, u);
+}
+__device__ __forceinline__ void store_out1(float* base, int64_t idx, float v) { base[idx] = v; }
+__device__ __forceinline__ void store_out1(__nv_bfloat16* base, int64_t idx, float v) {
+  base[idx] = __float2bfloat16_rn(v);
+}
+
+// ---- internal launchers (defined in the per-operator .cu files) ------------
+// Softmax with fp32 or bf16 output; x fp32 [rows, cols].
+pd_status launch_softmax(const float* x, void* y, bool y_is_bf16, int64_t rows, int64_t cols, cudaStream_t s);
+// LayerNorm with fp32 or bf16 output.
+pd_status launch_layernorm(const float* x, const float* gamma, const float* beta, void* y, bool y_is_bf16,
+                           int64_t rows, int64_t cols, float eps, cudaStream_t s);
+pd_status launch_bias_gelu_residual(const float* x, const float* bias, const float* r, float* out,
+                                    int64_t rows, int64_t cols, cudaStream_t s);
+
+
+// One (optionally batched) bf16 contraction with a fused epilogue:
+//   C[bo][bi][m,n] = epilogue(alpha * sum_k A[bo][bi][m,k] * B[bo][bi][k,n])
+//   epilogue(v)    = act(v + bias[n]) + residual[m,n]
+// The batch index has two levels (outer, inner) so that the per-head operands
+// of attention can be addressed inside the packed [tokens, 3*hidden] tensor.
+struct GemmProblem {
+  const void* A = nullptr;  // bf16 [M, K], row stride lda
+  const void* B = nullptr;  // bf16 [K, N] (b_is_nk false) or [N, K] (true), row stride ldb
+  void* C = nullptr;        // c_dtype [M, N], row stride ldc
+  int64_t M = 0, N = 0, K = 0, lda = 0, ldb = 0, ldc = 0;
+  bool b_is_nk = false;
+  pd_dtype c_dtype = PD_BF16;
+  int64_t batch_inner = 1, batch_outer = 1;
+  int64_t strideA_inner = 0, strideA_outer = 0, strideB_inner = 0, strideB_outer = 0;
+  int64_t strideC_inner = 0, strideC_outer = 0;
+  float alpha = 1.0f;
+  const float* bias = nullptr;               // fp32 [N] or null
+  bool gelu = false;                         // erf-form GELU after the bias
+  const __nv_bfloat16* residual = nullptr;   // bf16 [M, N], row stride ldr, or null (unbatched only)
+  int64_t ldr = 0;
+};
+pd_status launch_gemm(const GemmProblem& p, cudaStream_t s);
+
+}  // namespace pd

@@ -1,0 +1,137 @@
+// Row-wise softmax, fp32 in, fp32 or bf16 out.
+//
+//   y[i,j] = exp(x[i,j] - m_i) / sum_j exp(x[i,j] - m_i),  m_i = max_j x[i,j]
+//
+// HBM-bound: 8 bytes per element (4 when writing bf16).  Each row is read from
+// global memory exactly once into registers with 128-bit loads, reduced with
+// warp shuffles, and written once.
+//   * cols <= 1024            : one warp per row (up to 8 float4 per lane)
+//   * cols <= 16384           : one CTA of 512 threads per row (up to 8 float4 per thread)
+//   * anything else / ragged  : one CTA per row, three passes from global/L2
+#include "pd_common.cuh"
+
+namespace pd {
+namespace {
+
+#define kNegInf (-INFINITY)
+
+// One row held by THREADS_PER_ROW threads, VPT float4 each; threads of a row are
+// consecutive lanes.  THREADS_PER_ROW == 32: one warp per row, several rows per
+// CTA.  THREADS_PER_ROW == blockDim.x: one row per CTA.
+template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA, typename OutT>
+__global__ void __launch_bounds__(THREADS_PER_CTA)
+softmax_rows_in_registers(const float* __restrict__ x, OutT* __restrict__ y, int64_t rows, int cols) {
+  constexpr int ROWS_PER_CTA = THREADS_PER_CTA / THREADS_PER_ROW;
+  constexpr int NWARPS = THREADS_PER_ROW / 32;
+  __shared__ float scratch[2][NWARPS];
+  const int t = threadIdx.x % THREADS_PER_ROW;
+  const int cols4 = cols >> 2;
+  for (int64_t row = (int64_t)blockIdx.x * ROWS_PER_CTA + threadIdx.x / THREADS_PER_ROW; row < rows;
+       row += (int64_t)gridDim.x * ROWS_PER_CTA) {
+    const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
+    float4 v[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int c = t + i * THREADS_PER_ROW;
+      v[i] = (c < cols4) ? ld_stream(xr + c) : make_float4(kNegInf, kNegInf, kNegInf, kNegInf);
+    }
+    float m = kNegInf;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) m = fmaxf(m, fmaxf(fmaxf(v[i].x, v[i].y), fmaxf(v[i].z, v[i].w)));
+    m = block_reduce<NWARPS, true>(m, scratch, 0);
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      v[i].x = expf(v[i].x - m);
+      v[i].y = expf(v[i].y - m);
+      v[i].z = expf(v[i].z - m);
+      v[i].w = expf(v[i].w - m);
+      s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+    }
+    s = block_reduce<NWARPS, false>(s, scratch, 1);
+    const float inv = 1.0f / s;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int c = t + i * THREADS_PER_ROW;
+      if (c < cols4)
+        store_out4(y, row * cols4 + c, make_float4(v[i].x * inv, v[i].y * inv, v[i].z * inv, v[i].w * inv));
+    }
+    if constexpr (NWARPS > 1) __syncthreads();  // scratch is reused by the next row
+  }
+}
+
+// Any cols, any alignment: one CTA per row, scalar coalesced accesses, the row
+// is re-read from L2 for the second and third pass.
+template <typename OutT>
+__global__ void __launch_bounds__(256)
+softmax_rows_generic(const float* __restrict__ x, OutT* __restrict__ y, int64_t rows, int64_t cols) {
+  __shared__ float scratch[2][8];
+  for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+    const float* xr = x + row * cols;
+    float m = kNegInf;
+    for (int64_t j = threadIdx.x; j < cols; j += 256) m = fmaxf(m, xr[j]);
+    m = block_reduce<8, true>(m, scratch, 0);
+    float s = 0.f;
+    for (int64_t j = threadIdx.x; j < cols; j += 256) s += expf(xr[j] - m);
+    s = block_reduce<8, false>(s, scratch, 1);
+    const float inv = 1.0f / s;
+    for (int64_t j = threadIdx.x; j < cols; j += 256) store_out1(y, row * cols + j, expf(xr[j] - m) * inv);
+    __syncthreads();
+  }
+}
+
+template <int VPT, typename OutT>
+void launch_warp_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStream_t s) {
+  constexpr int kThreads = 256, kRowsPerCta = kThreads / 32;
+  const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
+  const int grid = (int)(ctas < (int64_t)sm_count() * 64 ? ctas : (int64_t)sm_count() * 64);
+  softmax_rows_in_registers<VPT, 32, kThreads, OutT><<<grid, kThreads, 0, s>>>(x, y, rows, cols);
+}
+
+template <int VPT, typename OutT>
+void launch_cta_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStream_t s) {
+  constexpr int kThreads = 512;
+  const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
+  softmax_rows_in_registers<VPT, kThreads, kThreads, OutT><<<grid, kThreads, 0, s>>>(x, y, rows, cols);
+}
+
+template <typename OutT>
+pd_status dispatch(const float* x, OutT* y, int64_t rows, int64_t cols, cudaStream_t s) {
+  const bool vec_ok = (cols % 4 == 0) && aligned16(x) && ((reinterpret_cast<uintptr_t>(y) & (sizeof(OutT) * 4 - 1)) == 0);
+  if (vec_ok && cols <= 1024) {
+    const int c = (int)cols;
+    if (c <= 128) launch_warp_rows<1>(x, y, rows, c, s);
+    else if (c <= 256) launch_warp_rows<2>(x, y, rows, c, s);
+    else if (c <= 512) launch_warp_rows<4>(x, y, rows, c, s);
+    else launch_warp_rows<8>(x, y, rows, c, s);
+  } else if (vec_ok && cols <= 16384) {
+    const int c = (int)cols;
+    if (c <= 2048) launch_cta_rows<1>(x, y, rows, c, s);
+    else if (c <= 4096) launch_cta_rows<2>(x, y, rows, c, s);
+    else if (c <= 8192) launch_cta_rows<4>(x, y, rows, c, s);
+    else launch_cta_rows<8>(x, y, rows, c, s);
+  } else {
+    const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
+    softmax_rows_generic<OutT><<<grid, 256, 0, s>>>(x, y, rows, cols);
+  }
+  return check_launch();
+}
+
+}  // namespace
+
+pd_status launch_softmax(const float* x, void* y, bool y_is_bf16, int64_t rows, int64_t cols, cudaStream_t s) {
+  if (y_is_bf16) return dispatch(x, static_cast<__nv_bfloat16*>(y), rows, cols, s);
+  return dispatch(x, static_cast<float*>(y), rows, cols, s);
+}
+
+}  // namespace pd
+
+extern "C" pd_status pd_softmax(const float* x, float* y, int64_t rows, int64_t cols, cudaStream_t stream) {
+  if (!x || !y) return PD_ERR_NULL_POINTER;
+  if (rows < 0 || cols <= 0) return PD_ERR_BAD_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y)) & 3u) return PD_ERR_ALIGNMENT;
+  if (rows == 0) return PD_OK;
+  pd_status st = pd::require_sm100();
+  if (st != PD_OK) return st;
+  return pd::launch_softmax(x, y, false, rows, cols, stream);
+}

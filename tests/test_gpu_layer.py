@@ -1,0 +1,85 @@
+"""GPU parity of pd_encoder_layer_fwd against the CPU oracle through the C ABI.
+Tolerance 2e-2 relative (denominator floored at the RMS of the oracle output):
+the bound for the bf16 layer, whose Q/K/V, probabilities, Ctx, H1 and Mid are
+stored in bf16 while the oracle rounds nothing."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_03586_b200 import inputs
+from parity import dev_bf16, dev_f32, host, max_rel_floored
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+_MATS = ("w_qkv", "w_o", "w_ffn1", "w_ffn2")
+_VECS = ("b_qkv", "b_o", "b_ffn1", "b_ffn2", "ln1_gamma", "ln1_beta", "ln2_gamma", "ln2_beta")
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2511_03586_b200 import api
+    api.pd_clear_device_status()
+    yield api
+    assert api.pd_get_device_status() == 0, "a bounded wait expired inside a tensor-core kernel"
+
+
+def _device_params(api, p):
+    kw = {m: dev_bf16(p[m + "_bits"]) for m in _MATS}
+    kw.update({v: dev_f32(p[v]) for v in _VECS})
+    return api.EncoderLayerParams(**kw)
+
+
+def _oracle_layer(p, shape, rows=slice(None), batch=None):
+    w = {m: inputs.bf16_bits_to_f32(p[m + "_bits"]) for m in _MATS}
+    x = inputs.bf16_bits_to_f32(p["x_bits"])[rows]
+    return oracle.encoder_layer(x, w["w_qkv"], p["b_qkv"], w["w_o"], p["b_o"], w["w_ffn1"], p["b_ffn1"],
+                                w["w_ffn2"], p["b_ffn2"], p["ln1_gamma"], p["ln1_beta"], p["ln2_gamma"],
+                                p["ln2_beta"], batch=shape.batch if batch is None else batch, seq=shape.seq,
+                                heads=shape.heads, ln_eps=np.float32(shape.ln_eps))
+
+
+@pytest.mark.parametrize("dims", [(2, 64, 2, 256), (3, 136, 1, 72), (1, 512, 4, 1024), (5, 8, 3, 8)])
+@pytest.mark.parametrize("w_sigma", [0.02, 0.08])
+def test_small_layers(api, dims, w_sigma):
+    batch, seq, heads, ffn = dims
+    shape = inputs.EncoderLayerShape(batch=batch, seq=seq, hidden=64 * heads, heads=heads, ffn=ffn)
+    p = inputs.encoder_layer_inputs(shape, seed=seq, w_sigma=w_sigma)
+    y = api.pd_encoder_layer_fwd(_device_params(api, p), dev_bf16(p["x_bits"]), batch=batch, seq=seq, heads=heads)
+    ref = _oracle_layer(p, shape)
+    assert max_rel_floored(host(y), ref) < TOL
+
+
+def test_bert_large_shape_sampled_sequences(api):
+    shape = inputs.EncoderLayerShape()                 # 32 x 512 tokens, hidden 1024, 16 heads, FFN 4096
+    p = inputs.encoder_layer_inputs(shape, seed=0)
+    params = _device_params(api, p)
+    x = dev_bf16(p["x_bits"])
+    nbytes = api.pd_encoder_layer_workspace_bytes(shape.batch, shape.seq, shape.hidden, shape.heads, shape.ffn)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    y = api.pd_encoder_layer_fwd(params, x, batch=shape.batch, seq=shape.seq, heads=shape.heads, workspace=ws)
+    y2 = api.pd_encoder_layer_fwd(params, x, batch=shape.batch, seq=shape.seq, heads=shape.heads, workspace=ws)
+    assert torch.equal(y, y2)                           # deterministic
+    assert bool(torch.isfinite(y.float()).all())
+    # sequences are independent, so the oracle is run on one of them (about 7 G multiply-adds)
+    b = 17
+    rows = slice(b * shape.seq, (b + 1) * shape.seq)
+    ref = _oracle_layer(p, shape, rows=rows, batch=1)
+    assert max_rel_floored(host(y[rows]), ref) < TOL
+    # property that holds at any size: every output row, un-affined, has zero mean and unit variance
+    g2, b2 = dev_f32(p["ln2_gamma"]), dev_f32(p["ln2_beta"])
+    z = (y.float() - b2) / g2
+    assert float(z.mean(dim=1).abs().max()) < 0.05
+    assert float((z.var(dim=1, unbiased=False) - 1).abs().max()) < 0.05
+
+
+def test_layer_argument_errors(api):
+    shape = inputs.EncoderLayerShape(batch=1, seq=16, hidden=64, heads=1, ffn=64)
+    p = inputs.encoder_layer_inputs(shape, seed=0)
+    params = _device_params(api, p)
+    x = dev_bf16(p["x_bits"])
+    with pytest.raises(api.PdError, match="PD_ERR_WORKSPACE_TOO_SMALL"):
+        api.pd_encoder_layer_fwd(params, x, batch=1, seq=16, heads=1, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(api.PdError, match="PD_ERR_UNSUPPORTED"):
+        api.pd_encoder_layer_fwd(params, x, batch=1, seq=16, heads=2)     # hidden != heads * 64

@@ -1,0 +1,140 @@
+"""GPU parity of pd_softmax / pd_layernorm / pd_bias_gelu_residual against the
+CPU oracle, called through the C ABI.  Tolerance: max relative error 1e-5 (fp32
+row operators); for outputs that end in an addition the denominator is floored
+at the RMS of the oracle tensor (see parity.max_rel_floored)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_03586_b200 import inputs
+from parity import Guarded, dev_f32, host, max_rel, max_rel_floored
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+ROWS = (1, 3, 33)
+COLS = (1, 2, 3, 4, 5, 31, 32, 33, 127, 128, 129, 512, 1000, 1024, 1028, 2048, 4096, 5000, 8192, 16384, 16388, 40000)
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2511_03586_b200 import api
+    return api
+
+
+@pytest.mark.parametrize("cols", COLS)
+def test_softmax_shapes(api, cols):
+    for rows in ROWS:
+        x = inputs.softmax_inputs(rows, cols, seed=rows)["x"]
+        y = Guarded((rows, cols), torch.float32)
+        api.pd_softmax(dev_f32(x), y.t)
+        torch.cuda.synchronize()
+        y.check()
+        assert max_rel(host(y.t), oracle.softmax(x)) < TOL
+
+
+def test_softmax_configured_and_paper_shapes(api):
+    for rows, cols in ((256, 512), (24576, 512)):
+        x = inputs.softmax_inputs(rows, cols, seed=0)["x"]
+        y = api.pd_softmax(dev_f32(x))
+        got = host(y)
+        assert max_rel(got, oracle.softmax(x)) < TOL
+        assert np.max(np.abs(got.sum(axis=1) - 1)) < 1e-5
+
+
+def test_softmax_in_place_unaligned_and_deterministic(api):
+    x = inputs.softmax_inputs(65, 516, seed=5)["x"]
+    xd = dev_f32(x)
+    y1 = api.pd_softmax(xd)
+    y2 = api.pd_softmax(xd)
+    assert torch.equal(y1, y2)
+    api.pd_softmax(xd, xd)
+    assert torch.equal(xd, y1)
+    # a view that starts 4 bytes into an allocation takes the scalar path
+    raw = torch.empty(65 * 516 + 1, dtype=torch.float32, device="cuda")
+    xu = raw[1:].view(65, 516)
+    xu.copy_(torch.from_numpy(x))
+    assert max_rel(host(api.pd_softmax(xu)), oracle.softmax(x)) < TOL
+    # constant rows give exactly 1/cols when cols is a power of two
+    c = torch.full((4, 256), 3.5, device="cuda")
+    assert torch.equal(api.pd_softmax(c), torch.full((4, 256), 1 / 256, device="cuda"))
+
+
+@pytest.mark.parametrize("cols", COLS)
+def test_layernorm_shapes(api, cols):
+    for rows in ROWS:
+        p = inputs.layernorm_inputs(rows, cols, seed=rows)
+        y = Guarded((rows, cols), torch.float32)
+        api.pd_layernorm(dev_f32(p["x"]), dev_f32(p["gamma"]), dev_f32(p["beta"]), p["eps"], y.t)
+        torch.cuda.synchronize()
+        y.check()
+        ref = oracle.layernorm(p["x"], p["gamma"], p["beta"], np.float32(p["eps"]))
+        if cols == 1:
+            assert np.allclose(host(y.t), ref, atol=1e-6)
+        else:
+            assert max_rel_floored(host(y.t), ref) < TOL
+
+
+def test_layernorm_configured_and_paper_shapes(api):
+    for rows, cols in ((4096, 1024), (16384, 1024), (4096, 4096)):
+        p = inputs.layernorm_inputs(rows, cols, seed=0)
+        xd = dev_f32(p["x"])
+        y = api.pd_layernorm(xd, dev_f32(p["gamma"]), dev_f32(p["beta"]), p["eps"])
+        ref = oracle.layernorm(p["x"], p["gamma"], p["beta"], np.float32(p["eps"]))
+        assert max_rel_floored(host(y), ref) < TOL
+        y2 = api.pd_layernorm(xd, dev_f32(p["gamma"]), dev_f32(p["beta"]), p["eps"], xd)   # in place
+        assert torch.equal(y, y2)
+
+
+def test_layernorm_large_mean_is_stable(api):
+    # mean >> spread: a one-pass E[x^2] - mu^2 variance would lose every digit here
+    rng = np.random.default_rng(9)
+    for cols in (1024, 4096, 40000):
+        x = (1000.0 + 0.01 * rng.standard_normal((3, cols))).astype(np.float32)
+        g, b = np.ones(cols, np.float32), np.zeros(cols, np.float32)
+        y = api.pd_layernorm(dev_f32(x), dev_f32(g), dev_f32(b), 0.0)
+        assert max_rel_floored(host(y), oracle.layernorm(x, g, b, 0.0)) < 1e-4
+
+
+@pytest.mark.parametrize("cols", COLS)
+def test_bias_gelu_residual_shapes(api, cols):
+    for rows in ROWS:
+        p = inputs.bias_gelu_residual_inputs(rows, cols, seed=rows)
+        out = Guarded((rows, cols), torch.float32)
+        api.pd_bias_gelu_residual(dev_f32(p["x"]), dev_f32(p["bias"]), dev_f32(p["r"]), out.t)
+        torch.cuda.synchronize()
+        out.check()
+        assert max_rel_floored(host(out.t), oracle.bias_gelu_residual(p["x"], p["bias"], p["r"])) < TOL
+        out2 = api.pd_bias_gelu_residual(dev_f32(p["x"]), dev_f32(p["bias"]), None)
+        assert max_rel_floored(host(out2), oracle.bias_gelu_residual(p["x"], p["bias"], None)) < TOL
+
+
+def test_bias_gelu_residual_configured_shape_sampled_rows(api):
+    rows, cols = 16384, 4096
+    p = inputs.bias_gelu_residual_inputs(rows, cols, seed=0)
+    xd, rd = dev_f32(p["x"]), dev_f32(p["r"])
+    out = api.pd_bias_gelu_residual(xd, dev_f32(p["bias"]), rd)
+    pick = np.unique(np.concatenate([[0, 1, rows - 1], np.random.default_rng(0).integers(0, rows, 200)]))
+    ref = oracle.bias_gelu_residual(p["x"][pick], p["bias"], p["r"][pick])
+    assert max_rel_floored(host(out[torch.from_numpy(pick).cuda()]), ref) < TOL
+    # wide range of arguments, including the far tails of erf
+    z = np.linspace(-12, 12, 4096 * 4, dtype=np.float32).reshape(4, 4096)
+    zero = np.zeros(4096, np.float32)
+    got = host(api.pd_bias_gelu_residual(dev_f32(z), dev_f32(zero), None))
+    assert np.max(np.abs(got - oracle.bias_gelu_residual(z, zero, None))) < 2e-6
+    # in place over x and over r
+    o1 = out.clone()
+    api.pd_bias_gelu_residual(xd, dev_f32(p["bias"]), rd, rd)
+    assert torch.equal(rd, o1)
+
+
+def test_rowop_errors(api):
+    x = torch.zeros(4, 8, device="cuda")
+    with pytest.raises(api.PdError, match="PD_ERR_BAD_SHAPE"):
+        api.pd_softmax(torch.zeros(4, 0, device="cuda"))
+    assert api.pd_softmax(torch.zeros(0, 8, device="cuda")).shape == (0, 8)
+    with pytest.raises(TypeError):
+        api.pd_softmax(x.double())
+    with pytest.raises(TypeError):
+        api.pd_softmax(x.cpu())
