@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the encoder-layer operator library on B200.
+
+One step = one forward pass of the BERT-large-shaped post-LN encoder layer
+(batch 32 x seq 512, hidden 1024, 16 heads, FFN 4096) through
+``pd_encoder_layer_fwd``: it runs every operator of the library (bf16 GEMMs with
+fused bias / GELU / residual epilogues, attention, softmax, LayerNorm) on one
+batch of seeded synthetic input.  The headline value is bf16 TFLOP/s counted
+over the six dense contractions (446.68 GFLOP per step).  The standalone
+operators at their configured and paper shapes are timed separately and
+reported under "ops" (GB/s for the row operators, TFLOP/s for the GEMM).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl pd|reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent
+replica on its own batch shard: the path has no exchange step, so there is no
+data-path collective; NCCL is used for the timing barrier and the max over ranks.
+``--impl reference`` times the CPU oracle (rank 0 only) on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2511_03586_b200 import inputs  # noqa: E402  (seeded generators only)
+
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+METRIC = "achieved HBM GB/s (row ops) and bf16 TFLOP/s (GEMM, layer) as % of roofline"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    except Exception:
+        return dict(FALLBACK_PEAKS, source="fallback")
+
+
+# ----------------------------------------------------------------------------
+# clocks during the timed region (NVML, read-only)
+# ----------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.index, self.period = index, period_s
+        self.sm, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._nv = None
+
+    def _sample(self):
+        try:
+            self.sm.append(int(self._nv.nvmlDeviceGetClockInfo(self._h, self._nv.NVML_CLOCK_SM)))
+            mask = int(self._nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+            for bit, name in self.REASONS.items():
+                if mask & bit and name != "gpu_idle":
+                    self.reasons.add(name)
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self._stop.is_set():
+            self._sample()
+            self._stop.wait(self.period)
+
+    def __enter__(self):
+        if self._nv:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        if self._thread:
+            self._sample()
+            self._stop.set()
+            self._thread.join()
+
+    def summary(self):
+        return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.sm)}
+
+
+# ----------------------------------------------------------------------------
+# CPU oracle legs
+# ----------------------------------------------------------------------------
+def oracle_layer_seconds(n_seq: int, seed: int = 0):
+    """Runs the CPU oracle's encoder layer on `n_seq` sequences of the workload; returns seconds."""
+    import oracle
+    shape = inputs.EncoderLayerShape(batch=n_seq)
+    p = inputs.encoder_layer_inputs(shape, seed=seed)
+    w = {m: inputs.bf16_bits_to_f32(p[m + "_bits"]) for m in ("w_qkv", "w_o", "w_ffn1", "w_ffn2")}
+    x = inputs.bf16_bits_to_f32(p["x_bits"])
+    oracle.softmax(np.zeros((1, 4)))  # load / build the library outside the timed part
+    t0 = time.perf_counter()
+    oracle.encoder_layer(x, w["w_qkv"], p["b_qkv"], w["w_o"], p["b_o"], w["w_ffn1"], p["b_ffn1"], w["w_ffn2"],
+                         p["b_ffn2"], p["ln1_gamma"], p["ln1_beta"], p["ln2_gamma"], p["ln2_beta"],
+                         batch=n_seq, seq=shape.seq, heads=shape.heads, ln_eps=shape.ln_eps)
+    return time.perf_counter() - t0, shape.gemm_flops()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    times = []
+    flops = 0.0
+    for i in range(args.warmup + args.steps):
+        dt, flops = oracle_layer_seconds(1, seed=i)
+        if i >= args.warmup:
+            times.append(dt)
+    sec = sum(times) / max(len(times), 1)
+    value = flops / sec / 1e12
+    sample = "one of the 32 sequences (batch 1 x seq 512) per step, full layer"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "bert-large post-LN encoder layer fwd, batch 32 x seq 512, hidden 1024, 16 heads, ffn 4096",
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": os.cpu_count()},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ----------------------------------------------------------------------------
+# GPU arm
+# ----------------------------------------------------------------------------
+def time_launches(torch, fn, n_iter, n_warm=3):
+    """Average device milliseconds of fn(i) over n_iter launches (CUDA events on the current stream)."""
+    for i in range(n_warm):
+        fn(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(n_iter):
+        fn(n_warm + i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / n_iter
+
+
+def ops_suite(torch, api, peaks, only: str = ""):
+    """Standalone operators at the configured and the paper's shapes.  Buffers rotate
+    through a pool larger than L2 so that every launch reads from HBM.  `only`
+    restricts the suite to the operators whose name contains it."""
+    out = {}
+    L2_POOL = 400 << 20
+
+    def wanted(name):
+        return only in name
+
+    def pool_size(bytes_per_set):
+        return max(2, min(256, -(-L2_POOL // bytes_per_set)))
+
+    def rowop_entry(name, ms, bytes_moved, note=None):
+        gbs = bytes_moved / ms / 1e6
+        e = {"ms": ms, "GB/s": gbs, "frac_measured": gbs / peaks["hbm_gbs"], "frac_nominal": gbs / NOMINAL_HBM_GBS}
+        if note:
+            e["note"] = note
+        out[name] = e
+
+    for rows, cols, note in ((256, 512, "configured shape: 1 MiB, launch-latency-bound"), (24576, 512, "paper shape"),
+                             (262144, 512, "attention rows of the layer")):
+        if not wanted(f"softmax_{rows}x{cols}"):
+            continue
+        x = torch.from_numpy(inputs.softmax_inputs(min(rows, 24576), cols)["x"]).cuda()
+        if rows > x.shape[0]:
+            x = x.repeat(-(-rows // x.shape[0]), 1)[:rows].contiguous()
+        n = pool_size(rows * cols * 8)
+        xs = [x.clone() for _ in range(n)]
+        ys = [torch.empty_like(x) for _ in range(n)]
+        iters = max(20, min(2000, int(3e9 / (rows * cols * 8))))
+        ms = time_launches(torch, lambda i: api.pd_softmax(xs[i % n], ys[i % n]), iters)
+        rowop_entry(f"softmax_{rows}x{cols}", ms, rows * cols * 8, note)
+        del xs, ys
+
+    for rows, cols, note in ((4096, 1024, "configured shape"), (16384, 1024, "paper shape"), (4096, 4096, "paper shape")):
+        if not wanted(f"layernorm_{rows}x{cols}"):
+            continue
+        p = inputs.layernorm_inputs(rows, cols)
+        x = torch.from_numpy(p["x"]).cuda()
+        g, b = torch.from_numpy(p["gamma"]).cuda(), torch.from_numpy(p["beta"]).cuda()
+        n = pool_size(rows * cols * 8)
+        xs = [x.clone() for _ in range(n)]
+        ys = [torch.empty_like(x) for _ in range(n)]
+        iters = max(20, min(2000, int(3e9 / (rows * cols * 8))))
+        ms = time_launches(torch, lambda i: api.pd_layernorm(xs[i % n], g, b, 1e-5, ys[i % n]), iters)
+        rowop_entry(f"layernorm_{rows}x{cols}", ms, rows * cols * 8 + cols * 8, note)
+        del xs, ys
+
+    rows, cols = 16384, 4096
+    if wanted(f"bias_gelu_residual_{rows}x{cols}"):
+        p = inputs.bias_gelu_residual_inputs(rows, cols)
+        xs = [torch.from_numpy(p["x"]).cuda() for _ in range(2)]
+        rs = [torch.from_numpy(p["r"]).cuda() for _ in range(2)]
+        os_ = [torch.empty_like(xs[0]) for _ in range(2)]
+        bias = torch.from_numpy(p["bias"]).cuda()
+        ms = time_launches(torch, lambda i: api.pd_bias_gelu_residual(xs[i % 2], bias, rs[i % 2], os_[i % 2]), 20)
+        rowop_entry(f"bias_gelu_residual_{rows}x{cols}", ms, rows * cols * 12 + cols * 4, "configured shape")
+        del xs, rs, os_, p
+
+    M, K, N = 16384, 1024, 4096
+    if not wanted(f"gemm_{M}x{N}x{K}"):
+        return out
+    g = inputs.gemm_inputs(M, N, K)
+    a = torch.from_numpy(g["a_bits"][0].view(np.int16)).cuda().view(torch.bfloat16)
+    b = torch.from_numpy(g["b_bits"][0].view(np.int16)).cuda().view(torch.bfloat16)
+    as_, bs = [a.clone() for _ in range(3)], [b.clone() for _ in range(3)]
+    for cd, nm in ((torch.bfloat16, "bf16"), (torch.float32, "f32")):
+        cs = [torch.empty(M, N, dtype=cd, device="cuda") for _ in range(3)]
+        ms = time_launches(torch, lambda i: api.pd_gemm_bf16(as_[i % 3], bs[i % 3], cs[i % 3]), 30)
+        tf = 2.0 * M * N * K / ms / 1e9
+        out[f"gemm_{M}x{N}x{K}_c{nm}"] = {"ms": ms, "TFLOP/s": tf, "frac_measured_burst": tf / peaks["bf16_tflops"],
+                                          "frac_measured_sustained": tf / peaks["bf16_tflops_sustained"],
+                                          "frac_nominal": tf / NOMINAL_BF16_TFLOPS, "note": "configured shape"}
+        del cs
+    return out
+
+
+def run_pd(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_2511_03586_b200 import api  # fails loudly when libpd.so is missing
+
+    peaks = load_peaks()
+    if args.ops_only:
+        if rank == 0:
+            print(json.dumps({"ops": ops_suite(torch, api, peaks, args.ops_filter), "peaks": peaks}), flush=True)
+        return 0
+    shape = inputs.EncoderLayerShape(batch=args.batch)
+    p = inputs.encoder_layer_inputs(shape, seed=rank)
+
+    def bf16_dev(bits):
+        return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    params = api.EncoderLayerParams(
+        **{m: bf16_dev(p[m + "_bits"]) for m in ("w_qkv", "w_o", "w_ffn1", "w_ffn2")},
+        **{v: torch.from_numpy(p[v]).cuda() for v in ("b_qkv", "b_o", "b_ffn1", "b_ffn2", "ln1_gamma", "ln1_beta",
+                                                       "ln2_gamma", "ln2_beta")})
+    x_host = torch.from_numpy(p["x_bits"].view(np.int16)).view(torch.bfloat16).pin_memory()
+    y_host = torch.empty_like(x_host).pin_memory()
+    x = x_host.cuda()
+    y = torch.empty_like(x)
+    ws = torch.empty(api.pd_encoder_layer_workspace_bytes(shape.batch, shape.seq, shape.hidden, shape.heads, shape.ffn),
+                     dtype=torch.uint8, device="cuda")
+    kw = dict(batch=shape.batch, seq=shape.seq, heads=shape.heads, ln_eps=shape.ln_eps, workspace=ws)
+    api.pd_clear_device_status()
+
+    def step():
+        api.pd_encoder_layer_fwd(params, x, y=y, **kw)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    # ---- device-resident throughput ------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+    barrier()
+    ms = e0.elapsed_time(e1) / args.steps
+
+    # ---- end to end: pinned host input -> device -> layer -> pinned host output --
+    def e2e_step():
+        x.copy_(x_host, non_blocking=True)
+        step()
+        y_host.copy_(y, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 50))
+    for _ in range(3):
+        e2e_step()
+    torch.cuda.synchronize()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, e2e_ms = float(t[0]), float(t[1])
+    timeout_code = api.pd_get_device_status()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    flops = shape.gemm_flops()
+    value = world * flops / ms / 1e9
+    stage_names = api.pd_encoder_layer_stage_names()
+
+    # ---- per-stage device times (CUDA events recorded by the library around each launch)
+    runs = []
+    for _ in range(7):
+        _, st = api.pd_encoder_layer_fwd_profiled(params, x, y=y, **kw)
+        runs.append(st)
+    stages = {n: statistics.median(r[n] for r in runs[2:]) for n in stage_names}
+
+    # dominant kernel: the tcgen05 GEMM; its largest launch is the FFN-up projection (= the configured GEMM shape)
+    T, H, F = shape.tokens, shape.hidden, shape.ffn
+    dom_flops = 2.0 * T * H * F
+    dom_tf = dom_flops / stages["ffn_up_gemm"] / 1e9
+    roofline = {"bound": "tensor", "kernel": "gemm_bf16_tcgen05_kernel<256,false> (ffn_up_gemm launch)",
+                "achieved": dom_tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": dom_tf / peaks["bf16_tflops_sustained"],
+                "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside the step)",
+                "frac_of_burst_peak": dom_tf / peaks["bf16_tflops"], "frac_of_nominal": dom_tf / NOMINAL_BF16_TFLOPS,
+                "traffic": None}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"bert-large post-LN encoder layer fwd, batch {shape.batch} x seq {shape.seq} per GPU, "
+                               f"hidden {shape.hidden}, {shape.heads} heads, ffn {shape.ffn} (configs[4])",
+                   "headline": "value = bf16 TFLOP/s of the whole layer step (six dense contractions); the row "
+                               "operators' GB/s and the standalone GEMM are under 'ops'",
+                   "flops_per_step_per_gpu": flops, "l2": "per-step working set (>1 GB) is larger than L2",
+                   "parallelism": "replicas only" if world > 1 else "single GPU", "sigma_reading": "N(a, b): b is the std"},
+        "frac_of_measured_sustained_peak": value / world / peaks["bf16_tflops_sustained"],
+        "frac_of_nominal_peak": value / world / NOMINAL_BF16_TFLOPS,
+        "clocks": clocks.summary(),
+        "e2e": {"value": world * flops / e2e_ms / 1e9, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": y_host.numel() * 2},
+        "gpu_launches": len(stage_names) * args.steps,
+        "device_timeout_code": timeout_code,
+        "stages_ms": stages,
+        "roofline": roofline,
+        "peaks": peaks,
+    }
+    if world == 1 and not args.no_ops:
+        line["ops"] = ops_suite(torch, api, peaks, args.ops_filter)
+    if world == 1 and not args.no_cpu_baseline:
+        n_seq = 2
+        sec, fl = oracle_layer_seconds(n_seq)
+        line["cpu_baseline"] = {"value": fl / sec / 1e12, "unit": "TFLOP/s", "cores": 1, "kind": "oracle",
+                                "sample": f"{n_seq} of the {shape.batch} sequences (batch {n_seq} x seq 512), full layer, "
+                                          f"{sec:.1f} s", "host_cores": os.cpu_count()}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=("pd", "reference"), default="pd")
+    ap.add_argument("--batch", type=int, default=32, help="sequences per GPU")
+    ap.add_argument("--no-ops", action="store_true", help="skip the standalone-operator suite")
+    ap.add_argument("--ops-only", action="store_true", help="run only the standalone-operator suite")
+    ap.add_argument("--ops-filter", default="", help="substring selecting operators of the suite")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_pd(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -142,6 +142,20 @@ pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, const pd_encod
                                const void* x, void* y, void* workspace, size_t workspace_bytes,
                                cudaStream_t stream);
 
+/* Measurement aid: the same forward pass with a CUDA event recorded around
+ * every stage the driver enqueues (the paper's evaluation likewise times each
+ * operator on its own, Section "Search with PerfLLM").  After enqueueing, the
+ * call WAITS for the layer to finish and writes the device time of stage i, in
+ * milliseconds, to stage_ms[i] (host pointer, pd_encoder_layer_stage_count()
+ * floats).  pd_encoder_layer_stage_name(i) names stage i (static storage, ""
+ * when out of range).  Results in y are identical to pd_encoder_layer_fwd. */
+int pd_encoder_layer_stage_count(void);
+const char* pd_encoder_layer_stage_name(int stage);
+pd_status pd_encoder_layer_fwd_profiled(const pd_encoder_layer_desc* desc,
+                                        const pd_encoder_layer_weights* weights, const void* x, void* y,
+                                        void* workspace, size_t workspace_bytes, cudaStream_t stream,
+                                        float* stage_ms);
+
 #ifdef __cplusplus
 }
 #endif

@@ -23,7 +23,8 @@ PD_BF16, PD_F32 = 0, 1
 EXPORTS = (
     "pd_status_string", "pd_last_cuda_error", "pd_get_device_status", "pd_clear_device_status",
     "pd_softmax", "pd_layernorm", "pd_bias_gelu_residual", "pd_gemm_bf16",
-    "pd_encoder_layer_workspace_bytes", "pd_encoder_layer_fwd",
+    "pd_encoder_layer_workspace_bytes", "pd_encoder_layer_fwd", "pd_encoder_layer_stage_count",
+    "pd_encoder_layer_stage_name", "pd_encoder_layer_fwd_profiled",
 )
 
 
@@ -66,6 +67,11 @@ def _load() -> ctypes.CDLL:
     lib.pd_encoder_layer_fwd.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.POINTER(EncoderLayerWeights),
                                          vp, vp, vp, ctypes.c_size_t, vp]
     lib.pd_encoder_layer_fwd.restype = st
+    lib.pd_encoder_layer_stage_count.argtypes = []; lib.pd_encoder_layer_stage_count.restype = ctypes.c_int
+    lib.pd_encoder_layer_stage_name.argtypes = [ctypes.c_int]
+    lib.pd_encoder_layer_stage_name.restype = ctypes.c_char_p
+    lib.pd_encoder_layer_fwd_profiled.argtypes = lib.pd_encoder_layer_fwd.argtypes + [ctypes.POINTER(ctypes.c_float)]
+    lib.pd_encoder_layer_fwd_profiled.restype = st
     return lib
 
 
@@ -196,6 +202,32 @@ def pd_encoder_layer_fwd(params: EncoderLayerParams, x: torch.Tensor, *, batch: 
                                      _dev(y, torch.bfloat16, "y"), workspace.data_ptr(), workspace.numel(),
                                      _stream(stream)), "pd_encoder_layer_fwd")
     return y
+
+
+def pd_encoder_layer_stage_names() -> list[str]:
+    return [_lib.pd_encoder_layer_stage_name(i).decode() for i in range(_lib.pd_encoder_layer_stage_count())]
+
+
+def pd_encoder_layer_fwd_profiled(params: EncoderLayerParams, x: torch.Tensor, *, batch: int, seq: int, heads: int,
+                                  ln_eps: float = 1e-5, y: torch.Tensor | None = None,
+                                  workspace: torch.Tensor | None = None, stream=None):
+    """Runs the layer with per-stage CUDA events; returns (y, {stage name: ms})."""
+    T, hidden = x.shape
+    if T != batch * seq:
+        raise ValueError("x must be [batch*seq, hidden]")
+    d = EncoderLayerDesc(batch, seq, hidden, heads, params.w_ffn1.shape[1], ln_eps)
+    if y is None:
+        y = torch.empty_like(x)
+    if workspace is None:
+        nbytes = int(_lib.pd_encoder_layer_workspace_bytes(ctypes.byref(d)))
+        workspace = torch.empty(max(nbytes, 1), dtype=torch.uint8, device=x.device)
+    w = params.as_struct()
+    n = _lib.pd_encoder_layer_stage_count()
+    ms = (ctypes.c_float * n)()
+    _check(_lib.pd_encoder_layer_fwd_profiled(ctypes.byref(d), ctypes.byref(w), _dev(x, torch.bfloat16, "x"),
+                                              _dev(y, torch.bfloat16, "y"), workspace.data_ptr(),
+                                              workspace.numel(), _stream(stream), ms), "pd_encoder_layer_fwd_profiled")
+    return y, dict(zip(pd_encoder_layer_stage_names(), [float(v) for v in ms]))
 
 
 def pd_get_device_status() -> int:

@@ -57,10 +57,22 @@ extern "C" size_t pd_encoder_layer_workspace_bytes(const pd_encoder_layer_desc* 
   return pd::plan(desc).total;
 }
 
-extern "C" pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* w,
-                                          const void* x, void* y, void* workspace, size_t workspace_bytes,
-                                          cudaStream_t stream) {
-  using namespace pd;
+namespace pd {
+namespace {
+
+constexpr int kStages = 9;
+const char* const kStageNames[kStages] = {"qkv_gemm", "scores_gemm", "softmax", "context_gemm", "out_proj_gemm",
+                                          "layernorm1", "ffn_up_gemm", "ffn_down_gemm", "layernorm2"};
+
+// Enqueues the whole layer.  When `ev` is not null it holds kStages + 1 events:
+// ev[i] is recorded before stage i and ev[kStages] after the last one.
+pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* w, const void* x, void* y,
+                    void* workspace, size_t workspace_bytes, cudaStream_t stream, cudaEvent_t* ev) {
+  int stage = 0;
+  auto mark = [&]() {
+    if (ev) cudaEventRecord(ev[stage], stream);
+    ++stage;
+  };
   if (!desc || !w || !x || !y) return PD_ERR_NULL_POINTER;
   if (!w->w_qkv || !w->w_o || !w->w_ffn1 || !w->w_ffn2 || !w->b_qkv || !w->b_o || !w->b_ffn1 || !w->b_ffn2 ||
       !w->ln1_gamma || !w->ln1_beta || !w->ln2_gamma || !w->ln2_beta)
@@ -90,12 +102,14 @@ extern "C" pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, con
   auto* mid = reinterpret_cast<__nv_bfloat16*>(base + ws.mid);
   const auto* xb = static_cast<const __nv_bfloat16*>(x);
 
+  mark();
   {  // QKV projection
     GemmProblem g;
     g.A = x; g.B = w->w_qkv; g.C = qkv; g.M = T; g.N = 3 * H; g.K = H; g.lda = H; g.ldb = 3 * H; g.ldc = 3 * H;
     g.bias = w->b_qkv;
     if ((st = launch_gemm(g, stream)) != PD_OK) return st;
   }
+  mark();
   {  // scores = Q K^T / sqrt(64), fp32, one [S, S] block per (batch, head)
     GemmProblem g;
     g.A = qkv; g.B = qkv + H; g.C = scores; g.M = S; g.N = S; g.K = kHeadDim; g.lda = 3 * H; g.ldb = 3 * H; g.ldc = S;
@@ -106,7 +120,9 @@ extern "C" pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, con
     g.strideC_inner = S * S; g.strideC_outer = NH * S * S;
     if ((st = launch_gemm(g, stream)) != PD_OK) return st;
   }
+  mark();
   if ((st = launch_softmax(scores, probs, true, B * NH * S, S, stream)) != PD_OK) return st;
+  mark();
   {  // Ctx = P V, heads written back to their column blocks
     GemmProblem g;
     g.A = probs; g.B = qkv + 2 * H; g.C = ctx; g.M = S; g.N = kHeadDim; g.K = S; g.lda = S; g.ldb = 3 * H; g.ldc = H;
@@ -116,24 +132,72 @@ extern "C" pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, con
     g.strideC_inner = kHeadDim; g.strideC_outer = S * H;
     if ((st = launch_gemm(g, stream)) != PD_OK) return st;
   }
+  mark();
   {  // output projection + bias + residual (fp32 sum kept for the LayerNorm)
     GemmProblem g;
     g.A = ctx; g.B = w->w_o; g.C = pre; g.M = T; g.N = H; g.K = H; g.lda = H; g.ldb = H; g.ldc = H;
     g.c_dtype = PD_F32; g.bias = w->b_o; g.residual = xb; g.ldr = H;
     if ((st = launch_gemm(g, stream)) != PD_OK) return st;
   }
+  mark();
   if ((st = launch_layernorm(pre, w->ln1_gamma, w->ln1_beta, h1, true, T, H, desc->ln_eps, stream)) != PD_OK) return st;
+  mark();
   {  // FFN up + bias + GELU
     GemmProblem g;
     g.A = h1; g.B = w->w_ffn1; g.C = mid; g.M = T; g.N = F; g.K = H; g.lda = H; g.ldb = F; g.ldc = F;
     g.bias = w->b_ffn1; g.gelu = true;
     if ((st = launch_gemm(g, stream)) != PD_OK) return st;
   }
+  mark();
   {  // FFN down + bias + residual
     GemmProblem g;
     g.A = mid; g.B = w->w_ffn2; g.C = pre; g.M = T; g.N = H; g.K = F; g.lda = F; g.ldb = H; g.ldc = H;
     g.c_dtype = PD_F32; g.bias = w->b_ffn2; g.residual = h1; g.ldr = H;
     if ((st = launch_gemm(g, stream)) != PD_OK) return st;
   }
-  return launch_layernorm(pre, w->ln2_gamma, w->ln2_beta, y, true, T, H, desc->ln_eps, stream);
+  mark();
+  st = launch_layernorm(pre, w->ln2_gamma, w->ln2_beta, y, true, T, H, desc->ln_eps, stream);
+  mark();
+  return st;
+}
+
+}  // namespace
+}  // namespace pd
+
+extern "C" pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* w,
+                                          const void* x, void* y, void* workspace, size_t workspace_bytes,
+                                          cudaStream_t stream) {
+  return pd::run_layer(desc, w, x, y, workspace, workspace_bytes, stream, nullptr);
+}
+
+extern "C" int pd_encoder_layer_stage_count(void) { return pd::kStages; }
+
+extern "C" const char* pd_encoder_layer_stage_name(int stage) {
+  return (stage >= 0 && stage < pd::kStages) ? pd::kStageNames[stage] : "";
+}
+
+extern "C" pd_status pd_encoder_layer_fwd_profiled(const pd_encoder_layer_desc* desc,
+                                                   const pd_encoder_layer_weights* w, const void* x, void* y,
+                                                   void* workspace, size_t workspace_bytes, cudaStream_t stream,
+                                                   float* stage_ms) {
+  using namespace pd;
+  if (!stage_ms) return PD_ERR_NULL_POINTER;
+  cudaEvent_t ev[kStages + 1];
+  int created = 0;
+  cudaError_t e = cudaSuccess;
+  for (; created <= kStages; ++created)
+    if ((e = cudaEventCreate(&ev[created])) != cudaSuccess) break;
+  pd_status st = e == cudaSuccess ? PD_OK : record_cuda_error(e);
+  if (st == PD_OK) st = run_layer(desc, w, x, y, workspace, workspace_bytes, stream, ev);
+  if (st == PD_OK) {
+    // an empty batch records nothing: report zeros
+    const bool ran = desc->batch > 0;
+    if (ran && (e = cudaEventSynchronize(ev[kStages])) != cudaSuccess) st = record_cuda_error(e);
+    for (int i = 0; i < kStages && st == PD_OK; ++i) {
+      stage_ms[i] = 0.f;
+      if (ran && (e = cudaEventElapsedTime(&stage_ms[i], ev[i], ev[i + 1])) != cudaSuccess) st = record_cuda_error(e);
+    }
+  }
+  for (int i = 0; i < created; ++i) cudaEventDestroy(ev[i]);
+  return st;
 }

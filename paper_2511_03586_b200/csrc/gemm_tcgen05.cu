@@ -152,8 +152,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
           if ((uint32_t)s >= issued) break;
           const uint32_t last = ((issued - 1 - s) / kStages) * kStages + s;
           volatile int never = 0;
-          int sink = 0;
-          mbar_wait(full_bar(s), (last / kStages) & 1u, &never, &sink, 0, 20000000ull);
+          mbar_wait(full_bar(s), (last / kStages) & 1u, &never, nullptr, 0, 20000000ull);
         }
       }
     }
@@ -191,8 +190,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         // Let every MMA already issued finish before tensor memory is freed.
         mma_commit(drain_bar);
         volatile int never = 0;
-        int sink = 0;
-        mbar_wait(drain_bar, 0, &never, &sink, 0, 20000000ull);
+        mbar_wait(drain_bar, 0, &never, nullptr, 0, 20000000ull);
       }
     }
   } else {

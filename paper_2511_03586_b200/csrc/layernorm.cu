@@ -93,10 +93,12 @@ layernorm_rows_generic(const float* __restrict__ x, const float* __restrict__ ga
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
     const float* xr = x + row * cols;
-    // per-thread Welford over a strided slice of the row
+    // per-thread Welford over a strided slice of the row, on data shifted by the
+    // row's first element so that a large common offset costs no precision
+    const float shift = xr[0];
     Moments m{0.f, 0.f, 0.f};
     for (int64_t j = threadIdx.x; j < cols; j += 256) {
-      const float v = xr[j];
+      const float v = xr[j] - shift;
       m.n += 1.f;
       const float d = v - m.mean;
       m.mean += d / m.n;
@@ -120,7 +122,7 @@ layernorm_rows_generic(const float* __restrict__ x, const float* __restrict__ ga
     __syncthreads();
     const float mu = stat[0], rstd = stat[1];
     for (int64_t j = threadIdx.x; j < cols; j += 256)
-      store_out1(y, row * cols + j, (xr[j] - mu) * rstd * gamma[j] + beta[j]);
+      store_out1(y, row * cols + j, ((xr[j] - shift) - mu) * rstd * gamma[j] + beta[j]);
     __syncthreads();
   }
 }

@@ -55,8 +55,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 
 // Bounded wait.  Returns true when the phase with `parity` has completed.  Gives
 // up (returns false) when another role has already raised *abort_flag or when
-// `limit_ns` elapse; in the latter case it raises the flag and records `code`
-// in *status (first writer wins) so that the host can see which wait expired.
+// `limit_ns` elapse; in the latter case it raises the flag and, when `status`
+// is not null, records `code` in *status (a global-memory word; first writer
+// wins) so that the host can see which wait expired.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
                                           int code, uint64_t limit_ns = 2000000000ull) {
   if (mbar_try_wait(bar, parity)) return true;
@@ -70,7 +71,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         t0 = now;
       } else if (now - t0 > limit_ns) {
         *abort_flag = 1;
-        atomicCAS(status, 0, code);
+        if (status != nullptr) atomicCAS(status, 0, code);
         return false;
       }
     }
