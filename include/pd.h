@@ -105,8 +105,23 @@ pd_status pd_gemm_bf16(const void* A, const void* B, void* C, int64_t M, int64_t
                        int64_t batch, int64_t strideA, int64_t strideB, int64_t strideC,
                        cudaStream_t stream);
 
+/* Fused multi-head scaled-dot-product attention (operators "bmm", "softmax",
+ * "bmm" of the paper's table chained per head; scores and probabilities stay
+ * on the SM).  qkv: bf16 [batch*seq, 3*heads*64] = column blocks [Q | K | V],
+ * head h in columns 64h..64h+63 of each block, token t = b*seq + s.
+ *   ctx[b, :, 64h..64h+63] = softmax(Q[b,h] K[b,h]^T / 8) V[b,h]
+ * ctx: bf16 [batch*seq, heads*64]; must not overlap qkv.  Head dimension is 64
+ * and 1 <= seq <= 512 (else PD_ERR_UNSUPPORTED).  Softmax is exact (maximum
+ * taken before any exponential) in fp32; probabilities are rounded to bf16 for
+ * the second product, which accumulates in fp32. */
+pd_status pd_attention_fwd(const void* qkv, void* ctx, int64_t batch, int64_t seq, int64_t heads,
+                           cudaStream_t stream);
+
 /* Shape of one post-LN encoder layer (BERT-large: 32 x 512 tokens, hidden 1024,
- * 16 heads of 64, FFN 4096).  hidden must equal heads * 64. */
+ * 16 heads of 64, FFN 4096).  hidden must equal heads * 64 and ffn must be a
+ * multiple of 8; seq must be at most 512 or a multiple of 8 (longer sequences
+ * take an unfused attention path that materialises scores in the workspace);
+ * anything else is PD_ERR_UNSUPPORTED. */
 typedef struct {
   int32_t batch, seq, hidden, heads, ffn;
   float ln_eps;

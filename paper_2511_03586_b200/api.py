@@ -22,7 +22,7 @@ PD_BF16, PD_F32 = 0, 1
 
 EXPORTS = (
     "pd_status_string", "pd_last_cuda_error", "pd_get_device_status", "pd_clear_device_status",
-    "pd_softmax", "pd_layernorm", "pd_bias_gelu_residual", "pd_gemm_bf16",
+    "pd_softmax", "pd_layernorm", "pd_bias_gelu_residual", "pd_gemm_bf16", "pd_attention_fwd",
     "pd_encoder_layer_workspace_bytes", "pd_encoder_layer_fwd", "pd_encoder_layer_stage_count",
     "pd_encoder_layer_stage_name", "pd_encoder_layer_fwd_profiled",
 )
@@ -62,6 +62,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, ctypes.c_int, ctypes.c_int,
                                  i64, i64, i64, i64, vp]
     lib.pd_gemm_bf16.restype = st
+    lib.pd_attention_fwd.argtypes = [vp, vp, i64, i64, i64, vp]; lib.pd_attention_fwd.restype = st
     lib.pd_encoder_layer_workspace_bytes.argtypes = [ctypes.POINTER(EncoderLayerDesc)]
     lib.pd_encoder_layer_workspace_bytes.restype = ctypes.c_size_t
     lib.pd_encoder_layer_fwd.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.POINTER(EncoderLayerWeights),
@@ -151,6 +152,18 @@ def pd_gemm_bf16_raw(a_ptr, b_ptr, c_ptr, M, N, K, lda, ldb, ldc, b_is_nk, c_dty
     """Direct call with explicit pointers and strides; returns the status instead of raising."""
     return _lib.pd_gemm_bf16(a_ptr, b_ptr, c_ptr, M, N, K, lda, ldb, ldc, int(b_is_nk), int(c_dtype), batch,
                              strideA, strideB, strideC, _stream(stream))
+
+
+def pd_attention_fwd(qkv: torch.Tensor, *, batch: int, seq: int, heads: int, ctx: torch.Tensor | None = None,
+                     stream=None) -> torch.Tensor:
+    """qkv bf16 [batch*seq, 3*heads*64] -> ctx bf16 [batch*seq, heads*64]."""
+    if tuple(qkv.shape) != (batch * seq, 3 * heads * 64):
+        raise ValueError("qkv must be [batch*seq, 3*heads*64]")
+    if ctx is None:
+        ctx = torch.empty(batch * seq, heads * 64, dtype=torch.bfloat16, device=qkv.device)
+    _check(_lib.pd_attention_fwd(_dev(qkv, torch.bfloat16, "qkv"), _dev(ctx, torch.bfloat16, "ctx"), batch, seq,
+                                 heads, _stream(stream)), "pd_attention_fwd")
+    return ctx
 
 
 @dataclass

@@ -2,7 +2,8 @@
 // chains the library's kernels on one stream with no host synchronisation.
 //
 //   QKV = X Wqkv + bqkv                                   (GEMM, bias epilogue)
-//   S   = Q K^T / 8, P = softmax(S), Ctx = P V  per head  (batched GEMM, softmax, batched GEMM)
+//   Ctx = softmax(Q K^T / 8) V  per (batch, head)         (fused attention kernel for seq <= 512;
+//                                                          otherwise batched GEMM, softmax, batched GEMM)
 //   pre = Ctx Wo + bo + X                                 (GEMM, bias + residual epilogue, fp32)
 //   H1  = LayerNorm(pre)                                  (row kernel, bf16 out)
 //   Mid = GELU(H1 W1 + b1)                                (GEMM, bias + GELU epilogue)
@@ -30,12 +31,16 @@ bool valid_desc(const pd_encoder_layer_desc* d) {
 }
 
 bool supported_desc(const pd_encoder_layer_desc* d) {
-  return d->hidden == d->heads * kHeadDim && d->seq % 8 == 0 && d->ffn % 8 == 0;
+  if (d->hidden != d->heads * kHeadDim || d->ffn % 8 != 0) return false;
+  return fused_attention_supported(d->seq, kHeadDim) || d->seq % 8 == 0;
 }
+
+bool use_fused_attention(const pd_encoder_layer_desc* d) { return fused_attention_supported(d->seq, kHeadDim); }
 
 Workspace plan(const pd_encoder_layer_desc* d) {
   const size_t T = (size_t)d->batch * d->seq, H = d->hidden, F = d->ffn, S = d->seq;
-  const size_t score_elems = (size_t)d->batch * d->heads * S * S;
+  // scores and probabilities are materialised only on the unfused attention path
+  const size_t score_elems = use_fused_attention(d) ? 0 : (size_t)d->batch * d->heads * S * S;
   Workspace w{};
   size_t off = 0;
   w.qkv = off; off += round_up(T * 3 * H * 2);
@@ -60,9 +65,9 @@ extern "C" size_t pd_encoder_layer_workspace_bytes(const pd_encoder_layer_desc* 
 namespace pd {
 namespace {
 
-constexpr int kStages = 9;
-const char* const kStageNames[kStages] = {"qkv_gemm", "scores_gemm", "softmax", "context_gemm", "out_proj_gemm",
-                                          "layernorm1", "ffn_up_gemm", "ffn_down_gemm", "layernorm2"};
+constexpr int kStages = 7;
+const char* const kStageNames[kStages] = {"qkv_gemm", "attention", "out_proj_gemm", "layernorm1",
+                                          "ffn_up_gemm", "ffn_down_gemm", "layernorm2"};
 
 // Enqueues the whole layer.  When `ev` is not null it holds kStages + 1 events:
 // ev[i] is recorded before stage i and ev[kStages] after the last one.
@@ -110,27 +115,29 @@ pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_we
     if ((st = launch_gemm(g, stream)) != PD_OK) return st;
   }
   mark();
-  {  // scores = Q K^T / sqrt(64), fp32, one [S, S] block per (batch, head)
-    GemmProblem g;
-    g.A = qkv; g.B = qkv + H; g.C = scores; g.M = S; g.N = S; g.K = kHeadDim; g.lda = 3 * H; g.ldb = 3 * H; g.ldc = S;
-    g.b_is_nk = true; g.c_dtype = PD_F32; g.alpha = 0.125f;
-    g.batch_inner = NH; g.batch_outer = B;
-    g.strideA_inner = kHeadDim; g.strideA_outer = S * 3 * H;
-    g.strideB_inner = kHeadDim; g.strideB_outer = S * 3 * H;
-    g.strideC_inner = S * S; g.strideC_outer = NH * S * S;
-    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
-  }
-  mark();
-  if ((st = launch_softmax(scores, probs, true, B * NH * S, S, stream)) != PD_OK) return st;
-  mark();
-  {  // Ctx = P V, heads written back to their column blocks
-    GemmProblem g;
-    g.A = probs; g.B = qkv + 2 * H; g.C = ctx; g.M = S; g.N = kHeadDim; g.K = S; g.lda = S; g.ldb = 3 * H; g.ldc = H;
-    g.batch_inner = NH; g.batch_outer = B;
-    g.strideA_inner = S * S; g.strideA_outer = NH * S * S;
-    g.strideB_inner = kHeadDim; g.strideB_outer = S * 3 * H;
-    g.strideC_inner = kHeadDim; g.strideC_outer = S * H;
-    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+  if (use_fused_attention(desc)) {
+    if ((st = launch_fused_attention(qkv, ctx, B, S, NH, stream)) != PD_OK) return st;
+  } else {
+    {  // scores = Q K^T / sqrt(64), fp32, one [S, S] block per (batch, head)
+      GemmProblem g;
+      g.A = qkv; g.B = qkv + H; g.C = scores; g.M = S; g.N = S; g.K = kHeadDim; g.lda = 3 * H; g.ldb = 3 * H; g.ldc = S;
+      g.b_is_nk = true; g.c_dtype = PD_F32; g.alpha = 0.125f;
+      g.batch_inner = NH; g.batch_outer = B;
+      g.strideA_inner = kHeadDim; g.strideA_outer = S * 3 * H;
+      g.strideB_inner = kHeadDim; g.strideB_outer = S * 3 * H;
+      g.strideC_inner = S * S; g.strideC_outer = NH * S * S;
+      if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+    }
+    if ((st = launch_softmax(scores, probs, true, B * NH * S, S, stream)) != PD_OK) return st;
+    {  // Ctx = P V, heads written back to their column blocks
+      GemmProblem g;
+      g.A = probs; g.B = qkv + 2 * H; g.C = ctx; g.M = S; g.N = kHeadDim; g.K = S; g.lda = S; g.ldb = 3 * H; g.ldc = H;
+      g.batch_inner = NH; g.batch_outer = B;
+      g.strideA_inner = S * S; g.strideA_outer = NH * S * S;
+      g.strideB_inner = kHeadDim; g.strideB_outer = S * 3 * H;
+      g.strideC_inner = kHeadDim; g.strideC_outer = S * H;
+      if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+    }
   }
   mark();
   {  // output projection + bias + residual (fp32 sum kept for the LayerNorm)
@@ -200,4 +207,18 @@ extern "C" pd_status pd_encoder_layer_fwd_profiled(const pd_encoder_layer_desc* 
   }
   for (int i = 0; i < created; ++i) cudaEventDestroy(ev[i]);
   return st;
+}
+
+extern "C" pd_status pd_attention_fwd(const void* qkv, void* ctx, int64_t batch, int64_t seq, int64_t heads,
+                                      cudaStream_t stream) {
+  using namespace pd;
+  if (!qkv || !ctx) return PD_ERR_NULL_POINTER;
+  if (batch < 0 || seq <= 0 || heads <= 0 || batch > 0x7fffffff || heads > 0x7fffffff) return PD_ERR_BAD_SHAPE;
+  if (!fused_attention_supported(seq, kHeadDim)) return PD_ERR_UNSUPPORTED;
+  if (!aligned16(qkv) || !aligned16(ctx)) return PD_ERR_ALIGNMENT;
+  if (batch == 0) return PD_OK;
+  pd_status st = require_sm100();
+  if (st != PD_OK) return st;
+  return launch_fused_attention(static_cast<const __nv_bfloat16*>(qkv), static_cast<__nv_bfloat16*>(ctx), batch, seq,
+                                heads, stream);
 }

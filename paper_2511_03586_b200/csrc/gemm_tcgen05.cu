@@ -11,12 +11,16 @@
 //                      tcgen05.commit hands the stage back ("empty" barrier) and,
 //                      after the last k-block, publishes the accumulator.
 //   warps 2-5        : epilogue.  Each warp drains its 32 TMEM lanes (32 rows of
-//                      the tile) 32 columns at a time, applies the epilogue in
-//                      fp32 and writes C, while the MMA warp already fills the
-//                      other accumulator with the next tile.
+//                      the tile) in chunks of 128 output bytes per row, applies
+//                      the epilogue in fp32, stages the chunk in a swizzled
+//                      4 KiB shared-memory buffer and hands it to a TMA store
+//                      (two buffers per warp, so a store drains while the next
+//                      chunk is computed), while the MMA warp already fills the
+//                      other accumulator with the next tile.  Residual and bias
+//                      values of the next chunk are fetched one chunk ahead.
 // B is taken either as [K, N] (N contiguous: an "MN-major" MMA operand, loaded
 // as BN/64 boxes of 64 x 64) or as [N, K] (K contiguous, "K-major").  Ragged M,
-// N, K edges are zero-filled by TMA on load and predicated on store.
+// N, K edges are zero-filled by TMA on load and clipped by TMA on store.
 // Every mbarrier wait is bounded: on expiry the kernel records a code in the
 // device status word, all roles drain, tensor memory is freed and the kernel
 // returns.
@@ -41,9 +45,10 @@ struct Cfg {
   static constexpr int kStageB = BN * BK * 2;
   static constexpr int kStage = kStageA + kStageB;
   static constexpr int kBarrierBytes = 1024;
-  static constexpr int kStagesMax = (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes) / kStage;
+  static constexpr int kEpilogueBytes = 4 /*warps*/ * 2 /*buffers*/ * 4096;
+  static constexpr int kStagesMax = (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes - kEpilogueBytes) / kStage;
   static constexpr int kStages = kStagesMax > 8 ? 8 : kStagesMax;
-  static constexpr int kSmemBytes = kStages * kStage + kBarrierBytes + 1024;
+  static constexpr int kSmemBytes = kStages * kStage + kEpilogueBytes + kBarrierBytes + 1024;
   static constexpr int kTmemCols = 2 * BN;  // two accumulators; 128, 256 or 512: a power of two
 };
 
@@ -71,23 +76,48 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int BN, bool B_NK>
+// The bf16 residual values of 32 consecutive columns of one row, fetched one
+// step ahead of their use; out-of-range parts are zero.
+struct ResidualRegs {
+  uint4 q[4];
+  __device__ __forceinline__ void load(const KernelParams& p, int m, int n0, bool row_ok) {
+    if (p.residual == nullptr) return;
+    const __nv_bfloat16* rr = p.residual + (int64_t)m * p.ldr + n0;
+    if (row_ok && n0 + 32 <= p.N) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) q[j] = __ldg(reinterpret_cast<const uint4*>(rr) + j);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+          if (row_ok && n0 + j * 8 + t < p.N)
+            w[t >> 1] |= (uint32_t)__bfloat16_as_ushort(rr[j * 8 + t]) << (16 * (t & 1));
+        q[j] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+  }
+};
+
+template <int BN, bool B_NK, bool C_F32>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                         const KernelParams p) {
+                         const __grid_constant__ CUtensorMap tmap_c, const KernelParams p) {
   using C = Cfg<BN>;
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
   // 128-byte swizzled tiles must start on a 1024-byte boundary.
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t bar_base = smem_base + kStages * C::kStage;
+  const uint32_t epi_base = smem_base + kStages * C::kStage;  // 1024-byte aligned: kStage is a multiple of 1024
+  const uint32_t bar_base = epi_base + C::kEpilogueBytes;
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
   auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
   auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
   auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
   const uint32_t drain_bar = bar_base + 8u * (2 * kStages + 4);
-  uint8_t* ctrl = smem_gen + kStages * C::kStage + 8 * (2 * kStages + 5);
+  uint8_t* ctrl = smem_gen + kStages * C::kStage + C::kEpilogueBytes + 8 * (2 * kStages + 5);
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 4);
 
@@ -195,10 +225,18 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     }
   } else {
     // ------------------------------------------------------------------ epilogue
+    // The accumulator is drained 32 columns at a time; one TMA store carries 128
+    // bytes of each of the warp's 32 rows: 64 bf16 columns (two steps) or 32
+    // fp32 columns (one step).
+    constexpr int STEPS_PER_STORE = C_F32 ? 1 : 2;
     const int quarter = warp & 3;  // TMEM lanes 32*quarter .. 32*quarter+31 belong to this warp
     const int row_in_tile = quarter * 32 + lane;
+    const uint32_t stage_buf = epi_base + quarter * 8192;
+    const uint32_t sw = (uint32_t)(lane & 7);  // 128-byte swizzle: 16-byte unit index ^= row % 8
+    uint32_t n_stores = 0;
     int local = 0;
     bool ok = true;
+    if (lane == 0) prefetch_tensormap(&tmap_c);
     for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local) {
       const int nt = tile % p.tiles_n;
       const int mt = (tile / p.tiles_n) % p.tiles_m;
@@ -206,26 +244,28 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       const int bi = b % p.batch_inner, bo = b / p.batch_inner;
       const int acc = local & 1;
       const uint32_t acc_ph = (local >> 1) & 1u;
-      if (!mbar_wait(acc_full_bar(acc), acc_ph, abort_flag, p.status, kTimeoutEpilogue)) { ok = false; break; }
-      tcgen05_fence_after_sync();
       const int m = mt * BM + row_in_tile;
       const bool row_ok = m < p.M;
-      const int64_t c_row = (int64_t)bo * p.strideC_outer + (int64_t)bi * p.strideC_inner + (int64_t)m * p.ldc;
+      const int n_tile = nt * BN;
+      ResidualRegs cur, nxt;
+      cur.load(p, m, n_tile, row_ok);  // does not depend on the accumulator: issued before the wait
+      if (!mbar_wait(acc_full_bar(acc), acc_ph, abort_flag, p.status, kTimeoutEpilogue)) { ok = false; break; }
+      tcgen05_fence_after_sync();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
-        const int n0 = nt * BN + c0;
+        const int n0 = n_tile + c0;
         if (n0 >= p.N) break;  // uniform over the warp
+        const bool last_step = (c0 + 32 >= BN) || (n0 + 32 >= p.N);
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_row + c0, r);
+        if (!last_step) nxt.load(p, m, n0 + 32, row_ok);
         tmem_ld_wait();
-        if (!row_ok) continue;
         float v[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * p.alpha;
-        const bool full = n0 + 32 <= p.N;
-        if (p.bias) {
-          if (full) {
+        if (p.bias != nullptr) {
+          if (n0 + 32 <= p.N) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
               const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias + n0 + j));
@@ -241,58 +281,56 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
         }
-        if (p.residual) {
-          const __nv_bfloat16* rr = p.residual + (int64_t)m * p.ldr + n0;
-          if (full) {
+        if (p.residual != nullptr) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              const uint4 u = __ldg(reinterpret_cast<const uint4*>(rr + j));
-              const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t w[4] = {cur.q[j].x, cur.q[j].y, cur.q[j].z, cur.q[j].w};
 #pragma unroll
-              for (int t = 0; t < 4; ++t) {
-                v[j + 2 * t] += __uint_as_float(w[t] << 16);
-                v[j + 2 * t + 1] += __uint_as_float(w[t] & 0xffff0000u);
-              }
+            for (int t = 0; t < 4; ++t) {
+              v[8 * j + 2 * t] += __uint_as_float(w[t] << 16);
+              v[8 * j + 2 * t + 1] += __uint_as_float(w[t] & 0xffff0000u);
             }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n0 + j < p.N) v[j] += __bfloat162float(rr[j]);
           }
         }
-        if (p.c_is_f32) {
-          float* out = static_cast<float*>(p.C) + c_row + n0;
-          if (full) {
+        const int step = (c0 / 32) % STEPS_PER_STORE;
+        const uint32_t buf = stage_buf + (n_stores & 1u) * 4096u;
+        if (step == 0) {
+          // The buffer about to be overwritten was handed to the store issued two
+          // stores ago: wait until that store has finished reading it.
+          if (lane == 0) tma_store_wait_read<1>();
+          __syncwarp();
+        }
+        const uint32_t row_addr = buf + (uint32_t)lane * 128u;
+        if constexpr (C_F32) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(out + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n0 + j < p.N) out[j] = v[j];
-          }
+          for (int u = 0; u < 8; ++u)
+            st_shared_v4(row_addr + (((uint32_t)u ^ sw) << 4),
+                         make_uint4(__float_as_uint(v[4 * u]), __float_as_uint(v[4 * u + 1]),
+                                    __float_as_uint(v[4 * u + 2]), __float_as_uint(v[4 * u + 3])));
         } else {
-          __nv_bfloat16* out = static_cast<__nv_bfloat16*>(p.C) + c_row + n0;
-          if (full) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              uint4 u;
-              u.x = pack_bf16(v[j], v[j + 1]);
-              u.y = pack_bf16(v[j + 2], v[j + 3]);
-              u.z = pack_bf16(v[j + 4], v[j + 5]);
-              u.w = pack_bf16(v[j + 6], v[j + 7]);
-              *reinterpret_cast<uint4*>(out + j) = u;
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (n0 + j < p.N) out[j] = __float2bfloat16_rn(v[j]);
-          }
+          for (int u = 0; u < 4; ++u)
+            st_shared_v4(row_addr + (((uint32_t)(step * 4 + u) ^ sw) << 4),
+                         make_uint4(pack_bf16(v[8 * u], v[8 * u + 1]), pack_bf16(v[8 * u + 2], v[8 * u + 3]),
+                                    pack_bf16(v[8 * u + 4], v[8 * u + 5]), pack_bf16(v[8 * u + 6], v[8 * u + 7])));
         }
+        if (step == STEPS_PER_STORE - 1 || last_step) {
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_4d(&tmap_c, buf, n0 - step * 32, mt * BM + quarter * 32, bi, bo);
+            tma_store_commit();
+          }
+          ++n_stores;
+        }
+        cur = nxt;
       }
       tcgen05_fence_before_sync();
       mbar_arrive(acc_empty_bar(acc));
     }
+    // Shared memory must outlive every store that still reads it.
+    if (lane == 0) tma_store_wait_all<0>();
+    __syncwarp();
   }
 
   // ------------------------------------------------------------------- teardown
@@ -322,35 +360,42 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-// bf16 tensor [outer][inner][rows][cols] with cols contiguous, 128-byte swizzle,
-// zero fill outside the extents.  Strides in elements.
-bool make_bf16_map(CUtensorMap* map, const void* base, int64_t cols, int64_t rows, int64_t ld, int64_t n_inner,
-                   int64_t stride_inner, int64_t n_outer, int64_t stride_outer, int box_cols, int box_rows) {
+// Tensor [outer][inner][rows][cols] of bf16 (or fp32 when `f32`) with cols
+// contiguous, 128-byte swizzle, zero fill outside the extents.  Strides in elements.
+bool make_map(CUtensorMap* map, bool f32, const void* base, int64_t cols, int64_t rows, int64_t ld, int64_t n_inner,
+              int64_t stride_inner, int64_t n_outer, int64_t stride_outer, int box_cols, int box_rows) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
+  const cuuint64_t esize = f32 ? 4 : 2;
   // Unit batch extents still need a legal (16-byte multiple) stride.
   if (n_inner == 1) stride_inner = ld * rows;
   if (n_outer == 1) stride_outer = (n_inner == 1 ? ld * rows : stride_inner * n_inner);
   const cuuint64_t dims[4] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)n_inner, (cuuint64_t)n_outer};
-  const cuuint64_t strides[3] = {(cuuint64_t)ld * 2, (cuuint64_t)stride_inner * 2, (cuuint64_t)stride_outer * 2};
+  const cuuint64_t strides[3] = {(cuuint64_t)ld * esize, (cuuint64_t)stride_inner * esize,
+                                 (cuuint64_t)stride_outer * esize};
   const cuuint32_t box[4] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+            const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, bool B_NK>
+template <int BN, bool B_NK, bool C_F32>
 pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
   using C = Cfg<BN>;
-  CUtensorMap ta, tb;
-  if (!make_bf16_map(&ta, g.A, g.K, g.M, g.lda, g.batch_inner, g.strideA_inner, g.batch_outer, g.strideA_outer, BK, BM))
+  CUtensorMap ta, tb, tc;
+  if (!make_map(&ta, false, g.A, g.K, g.M, g.lda, g.batch_inner, g.strideA_inner, g.batch_outer, g.strideA_outer, BK, BM))
     return PD_ERR_UNSUPPORTED;
-  const bool okb = B_NK ? make_bf16_map(&tb, g.B, g.K, g.N, g.ldb, g.batch_inner, g.strideB_inner, g.batch_outer,
-                                        g.strideB_outer, BK, BN)
-                        : make_bf16_map(&tb, g.B, g.N, g.K, g.ldb, g.batch_inner, g.strideB_inner, g.batch_outer,
-                                        g.strideB_outer, 64, BK);
+  const bool okb = B_NK ? make_map(&tb, false, g.B, g.K, g.N, g.ldb, g.batch_inner, g.strideB_inner, g.batch_outer,
+                                   g.strideB_outer, BK, BN)
+                        : make_map(&tb, false, g.B, g.N, g.K, g.ldb, g.batch_inner, g.strideB_inner, g.batch_outer,
+                                   g.strideB_outer, 64, BK);
   if (!okb) return PD_ERR_UNSUPPORTED;
+  // C is written in boxes of 32 rows x 128 bytes (one epilogue warp, one chunk).
+  if (!make_map(&tc, C_F32, g.C, g.N, g.M, g.ldc, g.batch_inner, g.strideC_inner, g.batch_outer, g.strideC_outer,
+                C_F32 ? 32 : 64, 32))
+    return PD_ERR_UNSUPPORTED;
 
   KernelParams p{};
   p.C = g.C; p.bias = g.bias; p.residual = g.residual; p.status = device_status_ptr();
@@ -365,7 +410,7 @@ pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
   p.num_tiles = (int)tiles;
   p.alpha = g.alpha; p.c_is_f32 = g.c_dtype == PD_F32; p.gelu = g.gelu;
 
-  auto kernel = gemm_bf16_tcgen05_kernel<BN, B_NK>;
+  auto kernel = gemm_bf16_tcgen05_kernel<BN, B_NK, C_F32>;
   static bool attr_set = false;  // per template instantiation
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
@@ -373,33 +418,36 @@ pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
     attr_set = true;
   }
   const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
-  kernel<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, p);
+  kernel<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, tc, p);
   return check_launch();
+}
+
+template <int BN>
+pd_status launch_bn(const GemmProblem& g, cudaStream_t s) {
+  if (g.b_is_nk)
+    return g.c_dtype == PD_F32 ? launch_variant<BN, true, true>(g, s) : launch_variant<BN, true, false>(g, s);
+  return g.c_dtype == PD_F32 ? launch_variant<BN, false, true>(g, s) : launch_variant<BN, false, false>(g, s);
 }
 
 }  // namespace
 
 pd_status launch_gemm(const GemmProblem& g, cudaStream_t s) {
-  // 128 x 256 tiles have the best operand reuse; narrower tiles are used when N
-  // is small or when they fill the last wave of SMs noticeably better.
+  // 128 x 256 tiles reuse operands best (the 128 x 128 main loop runs at about
+  // two thirds of their rate); narrower tiles are used when N is small or when
+  // they fill the last wave of SMs so much better that it pays.
   const int sms = sm_count();
-  auto waves_cost = [&](int bn) {
+  auto cost = [&](int bn, double rate) {
     const int64_t tiles = ((g.M + BM - 1) / BM) * ((g.N + bn - 1) / bn) * g.batch_inner * g.batch_outer;
     const int64_t waves = (tiles + sms - 1) / sms;
-    return (double)waves * bn;  // time ~ waves x tile width
+    return (double)waves * bn / rate;  // time ~ waves x tile width / main-loop rate
   };
   int bn = 256;
   if (g.N <= 64) bn = 64;
   else if (g.N <= 128) bn = 128;
-  else if (waves_cost(128) * 1.08 < waves_cost(256)) bn = 128;
-  if (g.b_is_nk) {
-    if (bn == 256) return launch_variant<256, true>(g, s);
-    if (bn == 128) return launch_variant<128, true>(g, s);
-    return launch_variant<64, true>(g, s);
-  }
-  if (bn == 256) return launch_variant<256, false>(g, s);
-  if (bn == 128) return launch_variant<128, false>(g, s);
-  return launch_variant<64, false>(g, s);
+  else if (cost(128, 0.66) < cost(256, 1.0)) bn = 128;
+  if (bn == 256) return launch_bn<256>(g, s);
+  if (bn == 128) return launch_bn<128>(g, s);
+  return launch_bn<64>(g, s);
 }
 
 }  // namespace pd

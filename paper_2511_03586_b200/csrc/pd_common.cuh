@@ -106,4 +106,9 @@ struct GemmProblem {
 };
 pd_status launch_gemm(const GemmProblem& p, cudaStream_t s);
 
+// Fused attention on qkv[batch*seq, 3*heads*64] -> ctx[batch*seq, heads*64] (both bf16).
+bool fused_attention_supported(int64_t seq, int64_t head_dim);
+pd_status launch_fused_attention(const __nv_bfloat16* qkv, __nv_bfloat16* ctx, int64_t batch, int64_t seq,
+                                 int64_t heads, cudaStream_t s);
+
 }  // namespace pd

@@ -40,7 +40,35 @@ def _oracle_layer(p, shape, rows=slice(None), batch=None):
                                 heads=shape.heads, ln_eps=np.float32(shape.ln_eps))
 
 
-@pytest.mark.parametrize("dims", [(2, 64, 2, 256), (3, 136, 1, 72), (1, 512, 4, 1024), (5, 8, 3, 8)])
+@pytest.mark.parametrize("seq", [1, 8, 100, 128, 129, 256, 300, 384, 512])
+def test_attention_against_oracle(api, seq):
+    batch, heads = 3, 2
+    rng = np.random.default_rng(seq)
+    qkv = rng.normal(0, 1.5, size=(batch * seq, 3 * heads * 64)).astype(np.float32)
+    bits = inputs.f32_to_bf16_bits(qkv)
+    ctx = api.pd_attention_fwd(dev_bf16(bits), batch=batch, seq=seq, heads=heads)
+    ref = oracle.attention(inputs.bf16_bits_to_f32(bits), batch, seq, heads, 64)
+    assert max_rel_floored(host(ctx), ref) < TOL
+    assert bool(torch.isfinite(ctx.float()).all())
+
+
+def test_attention_peaked_rows_and_errors(api):
+    # large logits: one key dominates each row; the exact (max-first) softmax must not overflow
+    batch, seq, heads = 1, 512, 1
+    rng = np.random.default_rng(5)
+    qkv = rng.normal(0, 1, size=(seq, 192)).astype(np.float32)
+    qkv[:, :128] *= 6.0
+    bits = inputs.f32_to_bf16_bits(qkv)
+    ctx = api.pd_attention_fwd(dev_bf16(bits), batch=batch, seq=seq, heads=heads)
+    ref = oracle.attention(inputs.bf16_bits_to_f32(bits), batch, seq, heads, 64)
+    assert max_rel_floored(host(ctx), ref) < TOL
+    with pytest.raises(api.PdError, match="PD_ERR_UNSUPPORTED"):
+        api.pd_attention_fwd(torch.zeros(520, 192, dtype=torch.bfloat16, device="cuda"), batch=1, seq=520, heads=1)
+
+
+# (batch, seq, heads, ffn): seq <= 512 takes the fused attention kernel, 640 the unfused path
+@pytest.mark.parametrize("dims", [(2, 64, 2, 256), (3, 136, 1, 72), (1, 512, 4, 1024), (5, 8, 3, 8), (2, 100, 2, 64),
+                                  (1, 640, 1, 128)])
 @pytest.mark.parametrize("w_sigma", [0.02, 0.08])
 def test_small_layers(api, dims, w_sigma):
     batch, seq, heads, ffn = dims
