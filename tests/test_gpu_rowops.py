@@ -131,9 +131,11 @@ def test_bias_gelu_residual_configured_shape_sampled_rows(api):
 
 def test_rowop_errors(api):
     x = torch.zeros(4, 8, device="cuda")
-    with pytest.raises(api.PdError, match="PD_ERR_BAD_SHAPE"):
-        api.pd_softmax(torch.zeros(4, 0, device="cuda"))
-    assert api.pd_softmax(torch.zeros(0, 8, device="cuda")).shape == (0, 8)
+    assert api._lib.pd_softmax(x.data_ptr(), x.data_ptr(), 4, 0, None) == 2        # cols == 0: PD_ERR_BAD_SHAPE
+    assert api._lib.pd_softmax(x.data_ptr(), x.data_ptr(), 0, 8, None) == 0        # rows == 0: PD_OK, no launch
+    assert api._lib.pd_softmax(x.data_ptr(), None, 4, 8, None) == 1                # PD_ERR_NULL_POINTER
+    with pytest.raises(api.PdError, match="PD_ERR_NULL_POINTER"):
+        api.pd_softmax(torch.zeros(4, 0, device="cuda"))                           # an empty tensor has no storage
     with pytest.raises(TypeError):
         api.pd_softmax(x.double())
     with pytest.raises(TypeError):
