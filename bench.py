@@ -38,6 +38,10 @@ from paper_2511_03586_b200 import inputs  # noqa: E402  (seeded generators only)
 NOMINAL_HBM_GBS = 8000.0
 NOMINAL_BF16_TFLOPS = 2250.0
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel at the FFN-up / configured
+# GEMM shape, from the ncu capture summarised in profiles/gemm_bf16_tcgen05_16384x4096x1024.md.  Set to None
+# whenever that kernel changes until the counters are taken again.
+DOMINANT_KERNEL_DRAM_TRAFFIC_BYTES = 42.008320e6 + 77.843200e6
 METRIC = "achieved HBM GB/s (row ops) and bf16 TFLOP/s (GEMM, layer) as % of roofline"
 
 
@@ -358,7 +362,7 @@ def run_pd(args):
                 "frac": dom_tf / peaks["bf16_tflops_sustained"],
                 "peak_source": f"{peaks['source']} sustained cuBLAS bf16 (kernel timed inside the step)",
                 "frac_of_burst_peak": dom_tf / peaks["bf16_tflops"], "frac_of_nominal": dom_tf / NOMINAL_BF16_TFLOPS,
-                "traffic": None}
+                "traffic": DOMINANT_KERNEL_DRAM_TRAFFIC_BYTES, "algorithmic_bytes": 2.0 * (T * H + H * F + T * F)}
 
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
