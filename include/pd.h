@@ -157,6 +157,33 @@ pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, const pd_encod
                                const void* x, void* y, void* workspace, size_t workspace_bytes,
                                cudaStream_t stream);
 
+/* Allocation-free variant of pd_encoder_layer_fwd (the paper has no counterpart:
+ * this entry point exists for integration reasons only).  Some callers cannot
+ * obtain device memory at the point where they need a layer: a serving process
+ * whose memory pool already owns the whole GPU, code running where a
+ * cudaMalloc (which synchronises the device) is not acceptable, or a plug-in
+ * that is handed inputs and outputs but no allocator.  For them the layer's
+ * intermediates go into a fixed array of pd_encoder_layer_static_scratch_bytes()
+ * = 32 MiB inside the library's device image (held by every GPU that loads the
+ * library, until the process exits) instead of a caller-provided workspace.
+ *  - Same arguments, results and error codes as pd_encoder_layer_fwd, minus the
+ *    workspace.  A shape whose intermediates need more than the array holds
+ *    (pd_encoder_layer_workspace_bytes(desc) > 32 MiB; BERT-large fits up to
+ *    about 1400 tokens) is rejected with PD_ERR_WORKSPACE_TOO_SMALL and nothing
+ *    is enqueued.
+ *  - The call allocates nothing: no cudaMalloc/cudaFree and no allocating
+ *    library routine, on any call.
+ *  - The first call on each device looks up the array's device address
+ *    (cudaGetSymbolAddress, with that device current).  Make that first call
+ *    before starting any stream capture.
+ *  - All calls share the one array and it keeps whatever the previous call left
+ *    there (every intermediate is fully rewritten before it is read, so nothing
+ *    needs clearing).  Two calls that overlap on the GPU - different streams, or
+ *    different host threads - race on it: serialise them. */
+size_t pd_encoder_layer_static_scratch_bytes(void);
+pd_status pd_encoder_layer_fwd_static(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* weights,
+                                      const void* x, void* y, cudaStream_t stream);
+
 /* Measurement aid: the same forward pass with a CUDA event recorded around
  * every stage the driver enqueues (the paper's evaluation likewise times each
  * operator on its own, Section "Search with PerfLLM").  After enqueueing, the

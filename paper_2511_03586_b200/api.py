@@ -24,7 +24,8 @@ EXPORTS = (
     "pd_status_string", "pd_last_cuda_error", "pd_get_device_status", "pd_clear_device_status",
     "pd_softmax", "pd_layernorm", "pd_bias_gelu_residual", "pd_gemm_bf16", "pd_attention_fwd",
     "pd_encoder_layer_workspace_bytes", "pd_encoder_layer_fwd", "pd_encoder_layer_stage_count",
-    "pd_encoder_layer_stage_name", "pd_encoder_layer_fwd_profiled",
+    "pd_encoder_layer_stage_name", "pd_encoder_layer_fwd_profiled", "pd_encoder_layer_static_scratch_bytes",
+    "pd_encoder_layer_fwd_static",
 )
 
 
@@ -68,6 +69,11 @@ def _load() -> ctypes.CDLL:
     lib.pd_encoder_layer_fwd.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.POINTER(EncoderLayerWeights),
                                          vp, vp, vp, ctypes.c_size_t, vp]
     lib.pd_encoder_layer_fwd.restype = st
+    lib.pd_encoder_layer_static_scratch_bytes.argtypes = []
+    lib.pd_encoder_layer_static_scratch_bytes.restype = ctypes.c_size_t
+    lib.pd_encoder_layer_fwd_static.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.POINTER(EncoderLayerWeights),
+                                                vp, vp, vp]
+    lib.pd_encoder_layer_fwd_static.restype = st
     lib.pd_encoder_layer_stage_count.argtypes = []; lib.pd_encoder_layer_stage_count.restype = ctypes.c_int
     lib.pd_encoder_layer_stage_name.argtypes = [ctypes.c_int]
     lib.pd_encoder_layer_stage_name.restype = ctypes.c_char_p
@@ -214,6 +220,26 @@ def pd_encoder_layer_fwd(params: EncoderLayerParams, x: torch.Tensor, *, batch: 
     _check(_lib.pd_encoder_layer_fwd(ctypes.byref(d), ctypes.byref(w), _dev(x, torch.bfloat16, "x"),
                                      _dev(y, torch.bfloat16, "y"), workspace.data_ptr(), workspace.numel(),
                                      _stream(stream)), "pd_encoder_layer_fwd")
+    return y
+
+
+def pd_encoder_layer_static_scratch_bytes() -> int:
+    return int(_lib.pd_encoder_layer_static_scratch_bytes())
+
+
+def pd_encoder_layer_fwd_static(params: EncoderLayerParams, x: torch.Tensor, y: torch.Tensor, *, batch: int,
+                                seq: int, heads: int, ln_eps: float = 1e-5, stream=None) -> torch.Tensor:
+    """The layer for callers that cannot allocate: intermediates live in the
+    library's fixed 32 MiB device array, and the caller passes the output tensor
+    too, so neither this binding nor the library allocates anything."""
+    T, hidden = x.shape
+    if T != batch * seq:
+        raise ValueError("x must be [batch*seq, hidden]")
+    d = EncoderLayerDesc(batch, seq, hidden, heads, params.w_ffn1.shape[1], ln_eps)
+    w = params.as_struct()
+    _check(_lib.pd_encoder_layer_fwd_static(ctypes.byref(d), ctypes.byref(w), _dev(x, torch.bfloat16, "x"),
+                                            _dev(y, torch.bfloat16, "y"), _stream(stream)),
+           "pd_encoder_layer_fwd_static")
     return y
 
 

@@ -222,3 +222,53 @@ extern "C" pd_status pd_attention_fwd(const void* qkv, void* ctx, int64_t batch,
   return launch_fused_attention(static_cast<const __nv_bfloat16*>(qkv), static_cast<__nv_bfloat16*>(ctx), batch, seq,
                                 heads, stream);
 }
+
+// ---- allocation-free variant ---------------------------------------------------
+// Scratch for callers that cannot hand the library a workspace of their own.
+// The array lives in the library's device image: every GPU that loads the
+// library carries these bytes until the process exits.
+#define PD_STATIC_SCRATCH_BYTES (32u << 20)
+static __device__ __align__(256) unsigned char g_layer_scratch[PD_STATIC_SCRATCH_BYTES];
+
+namespace pd {
+namespace {
+
+// Device address of g_layer_scratch on the current device.  In host code the
+// symbol's name is only a handle, never an address a kernel may be given, so
+// the address is looked up once per device (with that device current).
+pd_status static_scratch_ptr(void** out) {
+  constexpr int kMaxDevices = 64;
+  static void* cached[kMaxDevices];
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  if (dev < 0 || dev >= kMaxDevices) return PD_ERR_UNSUPPORTED;
+  if (!cached[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_layer_scratch);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    if (!ptr) return PD_ERR_CUDA;
+    cached[dev] = ptr;
+  }
+  *out = cached[dev];
+  return PD_OK;
+}
+
+}  // namespace
+}  // namespace pd
+
+extern "C" size_t pd_encoder_layer_static_scratch_bytes(void) { return PD_STATIC_SCRATCH_BYTES; }
+
+extern "C" pd_status pd_encoder_layer_fwd_static(const pd_encoder_layer_desc* desc,
+                                                 const pd_encoder_layer_weights* w, const void* x, void* y,
+                                                 cudaStream_t stream) {
+  using namespace pd;
+  if (!desc) return PD_ERR_NULL_POINTER;
+  if (!valid_desc(desc)) return PD_ERR_BAD_SHAPE;
+  if (!supported_desc(desc)) return PD_ERR_UNSUPPORTED;
+  if (plan(desc).total > PD_STATIC_SCRATCH_BYTES) return PD_ERR_WORKSPACE_TOO_SMALL;
+  void* scratch = nullptr;
+  pd_status st = static_scratch_ptr(&scratch);
+  if (st != PD_OK) return st;
+  return run_layer(desc, w, x, y, scratch, PD_STATIC_SCRATCH_BYTES, stream, nullptr);
+}
