@@ -2,7 +2,7 @@
 //
 //   C[m,n] = act(alpha * sum_k A[m,k] B[k,n] + bias[n]) + residual[m,n]
 //
-// Persistent, warp-specialised kernel, one CTA of 192 threads per SM:
+// Persistent, warp-specialised kernel, one CTA of 320 threads per SM:
 //   warp 0, one lane : TMA producer.  Streams 128 x 64 tiles of A and BN x 64
 //                      tiles of B (128-byte swizzle) into a ring of shared-memory
 //                      stages; a "full" mbarrier per stage counts the bytes.
@@ -10,14 +10,15 @@
 //                      accumulate into one of two TMEM accumulators; a
 //                      tcgen05.commit hands the stage back ("empty" barrier) and,
 //                      after the last k-block, publishes the accumulator.
-//   warps 2-5        : epilogue.  Each warp drains its 32 TMEM lanes (32 rows of
-//                      the tile) in chunks of 128 output bytes per row, applies
-//                      the epilogue in fp32, stages the chunk in a swizzled
-//                      4 KiB shared-memory buffer and hands it to a TMA store
-//                      (two buffers per warp, so a store drains while the next
-//                      chunk is computed), while the MMA warp already fills the
-//                      other accumulator with the next tile.  Residual and bias
-//                      values of the next chunk are fetched one chunk ahead.
+//   warps 2-9        : epilogue.  Two warps share each group of 32 TMEM lanes (32
+//                      rows of the tile) and take alternate chunks of 128 output
+//                      bytes per row.  A warp drains its chunk 32 columns at a
+//                      time (tcgen05.ld), applies the epilogue in fp32, stages
+//                      the chunk in its swizzled 4 KiB shared-memory buffer and
+//                      hands it to a TMA store, while its sibling works on the
+//                      next chunk and the MMA warp already fills the other
+//                      accumulator with the next tile.  Residual values are
+//                      fetched one step ahead.
 // B is taken either as [K, N] (N contiguous: an "MN-major" MMA operand, loaded
 // as BN/64 boxes of 64 x 64) or as [N, K] (K contiguous, "K-major").  Ragged M,
 // N, K edges are zero-filled by TMA on load and clipped by TMA on store.
@@ -35,8 +36,9 @@ using namespace sm100;
 constexpr int BM = 128;       // tile rows = TMEM lanes
 constexpr int BK = 64;        // k-block: 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;    // k extent of one tcgen05.mma for 16-bit inputs
-constexpr int kThreads = 192;
-constexpr int kEpilogueThreads = 128;
+constexpr int kEpilogueWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpilogueWarps;
+constexpr int kEpilogueThreads = 32 * kEpilogueWarps;
 constexpr int kSmemLimit = 227 * 1024;
 
 template <int BN>
@@ -45,7 +47,7 @@ struct Cfg {
   static constexpr int kStageB = BN * BK * 2;
   static constexpr int kStage = kStageA + kStageB;
   static constexpr int kBarrierBytes = 1024;
-  static constexpr int kEpilogueBytes = 4 /*warps*/ * 2 /*buffers*/ * 4096;
+  static constexpr int kEpilogueBytes = kEpilogueWarps * 4096;  // one 32-row x 128-byte staging buffer per warp
   static constexpr int kStagesMax = (kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes - kEpilogueBytes) / kStage;
   static constexpr int kStages = kStagesMax > 8 ? 8 : kStagesMax;
   static constexpr int kSmemBytes = kStages * kStage + kEpilogueBytes + kBarrierBytes + 1024;
@@ -67,8 +69,26 @@ struct KernelParams {
 // Codes left in the device status word by an expired wait.
 enum : int { kTimeoutProducer = 101, kTimeoutMmaFull = 102, kTimeoutMmaAcc = 103, kTimeoutEpilogue = 104 };
 
+// GELU in its erf form, z * Phi(z), with the normal tail evaluated as
+//   q = 2^P(t) ~ Phi(-t),  t = min(|z|, 5),  Phi(z) = z < 0 ? q : 1 - q,  q = 0 beyond 5.
+// P is the degree-6 minimax fit of log2 Phi(-t) on [0, 5] produced by
+// fit_gelu_tail_poly.py (max |dP| = 1.8e-5, i.e. a relative error of 1.2e-5 in the
+// tail; in fp32 the whole function stays within 1.5e-5 relative, 2e-6 absolute).
+// One exponential and ten FP32 operations per value instead of erff's branches.
 __device__ __forceinline__ float gelu_erf(float z) {
-  return 0.5f * z * (1.0f + erff(z * 0.70710678118654752440f));
+  const float a = fabsf(z);
+  const float t = fminf(a, 5.0f);
+  float p = 2.945814984e-05f;
+  p = fmaf(p, t, -7.087827801e-04f);
+  p = fmaf(p, t, 7.746013990e-03f);
+  p = fmaf(p, t, -5.260629289e-02f);
+  p = fmaf(p, t, -4.596254617e-01f);
+  p = fmaf(p, t, -1.150867236e+00f);
+  p = fmaf(p, t, -1.000017644e+00f);
+  float q;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(q) : "f"(p));
+  q = a > 5.0f ? 0.0f : q;
+  return z * (z < 0.0f ? q : 1.0f - q);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -226,14 +246,20 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   } else {
     // ------------------------------------------------------------------ epilogue
     // The accumulator is drained 32 columns at a time; one TMA store carries 128
-    // bytes of each of the warp's 32 rows: 64 bf16 columns (two steps) or 32
-    // fp32 columns (one step).
-    constexpr int STEPS_PER_STORE = C_F32 ? 1 : 2;
-    const int quarter = warp & 3;  // TMEM lanes 32*quarter .. 32*quarter+31 belong to this warp
+    // bytes of each of the warp's 32 rows: a chunk of 64 bf16 columns (two
+    // steps) or 32 fp32 columns (one step).  The two warps of a lane group take
+    // alternate chunks.
+    constexpr int STEPS = C_F32 ? 1 : 2;
+    constexpr int CW = 32 * STEPS;       // chunk width in columns
+    constexpr int NCHUNK = BN / CW;
+    const int quarter = warp & 3;         // TMEM lanes 32*quarter .. 32*quarter+31 belong to this warp
+    const int group = (warp - 2) >> 2;    // 0: even chunks, 1: odd chunks
     const int row_in_tile = quarter * 32 + lane;
-    const uint32_t stage_buf = epi_base + quarter * 8192;
+    const uint32_t buf = epi_base + (uint32_t)(warp - 2) * 4096u;
+    const uint32_t row_addr = buf + (uint32_t)lane * 128u;
     const uint32_t sw = (uint32_t)(lane & 7);  // 128-byte swizzle: 16-byte unit index ^= row % 8
-    uint32_t n_stores = 0;
+    const int my_steps = ((NCHUNK - group + 1) / 2) * STEPS;
+    auto col_of = [&](int i) { return ((i / STEPS) * 2 + group) * CW + (i % STEPS) * 32; };
     int local = 0;
     bool ok = true;
     if (lane == 0) prefetch_tensormap(&tmap_c);
@@ -248,18 +274,21 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       const bool row_ok = m < p.M;
       const int n_tile = nt * BN;
       ResidualRegs cur, nxt;
-      cur.load(p, m, n_tile, row_ok);  // does not depend on the accumulator: issued before the wait
+      if (my_steps > 0 && n_tile + col_of(0) < p.N)
+        cur.load(p, m, n_tile + col_of(0), row_ok);  // independent of the accumulator: issued before the wait
       if (!mbar_wait(acc_full_bar(acc), acc_ph, abort_flag, p.status, kTimeoutEpilogue)) { ok = false; break; }
       tcgen05_fence_after_sync();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
 #pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
+      for (int i = 0; i < my_steps; ++i) {
+        const int c0 = col_of(i);
         const int n0 = n_tile + c0;
-        if (n0 >= p.N) break;  // uniform over the warp
-        const bool last_step = (c0 + 32 >= BN) || (n0 + 32 >= p.N);
+        if (n0 >= p.N) break;  // uniform over the warp; columns grow with i
+        const int step = i % STEPS;
+        const bool has_next = (i + 1 < my_steps) && (n_tile + col_of(i + 1) < p.N);
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_row + c0, r);
-        if (!last_step) nxt.load(p, m, n0 + 32, row_ok);
+        if (has_next) nxt.load(p, m, n_tile + col_of(i + 1), row_ok);
         tmem_ld_wait();
         float v[32];
 #pragma unroll
@@ -292,15 +321,11 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
             }
           }
         }
-        const int step = (c0 / 32) % STEPS_PER_STORE;
-        const uint32_t buf = stage_buf + (n_stores & 1u) * 4096u;
         if (step == 0) {
-          // The buffer about to be overwritten was handed to the store issued two
-          // stores ago: wait until that store has finished reading it.
-          if (lane == 0) tma_store_wait_read<1>();
+          // the previous store of this warp must have finished reading the buffer
+          if (lane == 0) tma_store_wait_read<0>();
           __syncwarp();
         }
-        const uint32_t row_addr = buf + (uint32_t)lane * 128u;
         if constexpr (C_F32) {
 #pragma unroll
           for (int u = 0; u < 8; ++u)
@@ -314,14 +339,13 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
                          make_uint4(pack_bf16(v[8 * u], v[8 * u + 1]), pack_bf16(v[8 * u + 2], v[8 * u + 3]),
                                     pack_bf16(v[8 * u + 4], v[8 * u + 5]), pack_bf16(v[8 * u + 6], v[8 * u + 7])));
         }
-        if (step == STEPS_PER_STORE - 1 || last_step) {
+        if (step == STEPS - 1 || n0 + 32 >= p.N) {
           fence_proxy_async_smem();
           __syncwarp();
           if (lane == 0) {
             tma_store_4d(&tmap_c, buf, n0 - step * 32, mt * BM + quarter * 32, bi, bo);
             tma_store_commit();
           }
-          ++n_stores;
         }
         cur = nxt;
       }
