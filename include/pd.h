@@ -105,6 +105,16 @@ pd_status pd_gemm_bf16(const void* A, const void* B, void* C, int64_t M, int64_t
                        int64_t batch, int64_t strideA, int64_t strideB, int64_t strideC,
                        cudaStream_t stream);
 
+/* Tuning and testing aid for every contraction the library launches (it has no
+ * counterpart in the paper).  mode 0 (default): choose automatically between
+ * 128 x BN tiles computed by one CTA and 256 x 256 tiles computed by a pair of
+ * CTAs (tcgen05 cta_group::2); mode 1: single-CTA tiles only; mode 2: CTA-pair
+ * tiles for every shape.  Results do not depend on the mode beyond fp32
+ * summation order inside the tensor core (identical here: both walk k in
+ * ascending 16-element steps).  Process-wide, not thread-safe against
+ * concurrent launches.  Other values: PD_ERR_BAD_SHAPE. */
+pd_status pd_set_gemm_tile_mode(int mode);
+
 /* Fused multi-head scaled-dot-product attention (operators "bmm", "softmax",
  * "bmm" of the paper's table chained per head; scores and probabilities stay
  * on the SM).  qkv: bf16 [batch*seq, 3*heads*64] = column blocks [Q | K | V],

@@ -22,7 +22,7 @@ PD_BF16, PD_F32 = 0, 1
 
 EXPORTS = (
     "pd_status_string", "pd_last_cuda_error", "pd_get_device_status", "pd_clear_device_status",
-    "pd_softmax", "pd_layernorm", "pd_bias_gelu_residual", "pd_gemm_bf16", "pd_attention_fwd",
+    "pd_softmax", "pd_layernorm", "pd_bias_gelu_residual", "pd_gemm_bf16", "pd_set_gemm_tile_mode", "pd_attention_fwd",
     "pd_encoder_layer_workspace_bytes", "pd_encoder_layer_fwd", "pd_encoder_layer_stage_count",
     "pd_encoder_layer_stage_name", "pd_encoder_layer_fwd_profiled", "pd_encoder_layer_static_scratch_bytes",
     "pd_encoder_layer_fwd_static",
@@ -63,6 +63,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, ctypes.c_int, ctypes.c_int,
                                  i64, i64, i64, i64, vp]
     lib.pd_gemm_bf16.restype = st
+    lib.pd_set_gemm_tile_mode.argtypes = [ctypes.c_int]; lib.pd_set_gemm_tile_mode.restype = st
     lib.pd_attention_fwd.argtypes = [vp, vp, i64, i64, i64, vp]; lib.pd_attention_fwd.restype = st
     lib.pd_encoder_layer_workspace_bytes.argtypes = [ctypes.POINTER(EncoderLayerDesc)]
     lib.pd_encoder_layer_workspace_bytes.restype = ctypes.c_size_t
@@ -151,6 +152,11 @@ def pd_gemm_bf16(a: torch.Tensor, b: torch.Tensor, c: torch.Tensor | None = None
                              M, N, K, K, ldb, N, int(b_is_nk), PD_F32 if c.dtype == torch.float32 else PD_BF16,
                              batch, M * K, b.shape[-2] * b.shape[-1], M * N, _stream(stream)), "pd_gemm_bf16")
     return c
+
+
+def pd_set_gemm_tile_mode(mode: int) -> None:
+    """0: automatic; 1: single-CTA tiles only; 2: CTA-pair (cta_group::2) tiles for every shape."""
+    _check(_lib.pd_set_gemm_tile_mode(int(mode)), "pd_set_gemm_tile_mode")
 
 
 def pd_gemm_bf16_raw(a_ptr, b_ptr, c_ptr, M, N, K, lda, ldb, ldc, b_is_nk, c_dtype, batch, strideA, strideB,

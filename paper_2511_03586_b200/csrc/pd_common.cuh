@@ -105,6 +105,10 @@ struct GemmProblem {
   int64_t ldr = 0;
 };
 pd_status launch_gemm(const GemmProblem& p, cudaStream_t s);
+// The same contraction on 256 x 256 tiles computed by pairs of CTAs (cta_group::2).
+bool gemm_pair_tiles_profitable(const GemmProblem& p);
+void set_gemm_tile_mode(int mode);
+pd_status launch_gemm_pair(const GemmProblem& p, cudaStream_t s);
 
 // Fused attention on qkv[batch*seq, 3*heads*64] -> ctx[batch*seq, heads*64] (both bf16).
 bool fused_attention_supported(int64_t seq, int64_t head_dim);

@@ -17,11 +17,14 @@ pytestmark = pytest.mark.gpu
 TOL = 2e-2
 
 
-@pytest.fixture(scope="module")
-def api():
+@pytest.fixture(scope="module", params=[1, 2, 0], ids=["single_cta_tiles", "cta_pair_tiles", "auto_tiles"])
+def api(request):
+    """Every test runs with 128 x BN single-CTA tiles, with 256 x 256 CTA-pair tiles, and with the automatic choice."""
     from paper_2511_03586_b200 import api
     api.pd_clear_device_status()
+    api.pd_set_gemm_tile_mode(request.param)
     yield api
+    api.pd_set_gemm_tile_mode(0)
     assert api.pd_get_device_status() == 0, "a bounded wait expired inside a tensor-core kernel"
 
 
