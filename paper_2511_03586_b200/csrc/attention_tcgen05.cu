@@ -5,36 +5,49 @@
 // on the packed projection qkv[tokens, 3*hidden] = [Q | K | V].  Scores and
 // probabilities never leave the SM.
 //
-// One persistent CTA of 320 threads per SM walks over work units of
-// (batch, head, pair of 128-query blocks):
-//   warp 8, one lane : TMA producer.  K and V of the head (up to 512 x 64 each)
-//                      are loaded once per unit, Q once per query block.
-//   warp 9, one lane : MMA issuer.  S = Q K^T as one 128 x 128 x 64 product per
-//                      block of 128 keys into tensor memory (all 512 columns
-//                      hold the fp32 scores of the 128 queries), then, as the
-//                      softmax warps publish blocks of probabilities,
-//                      O += P_j V_j (128 x 64 x 128) into columns 0-63, which
-//                      the scores of block 0 no longer need by then.
-//   warps 0-7        : softmax, two threads per query row (warps 0-3 take the even
-//                      key blocks, warps 4-7 the odd ones).  Pass 1 reads the
-//                      scores from tensor memory and takes the row maximum
-//                      (the two halves exchange theirs through shared memory);
-//                      pass 2 re-reads them block by block, forms
-//                      p = 2^((s - max) * log2(e) / 8) (exact softmax: the maximum is
-//                      known before the first exponential, nothing is ever
-//                      rescaled), accumulates the fp32 row sum and writes P as
-//                      bf16 into the half's swizzled shared-memory tile, which
-//                      the MMA reads as its A operand.  Tensor-memory loads are
-//                      issued one chunk ahead of the arithmetic.  Finally each
-//                      thread reads 32 columns of its O row, divides by the row
-//                      sum and stores 32 bf16 values (64 contiguous bytes).
-// Keys beyond the sequence length are zero-filled by TMA and masked to -inf;
-// query rows beyond it are computed and discarded.
+// One persistent CTA of 416 threads per SM walks over work units of (batch,
+// head, pair of 128-query blocks).  K and V of the head (up to 512 x 64 each)
+// are resident in shared memory for the unit; the two query blocks ("slots")
+// are in flight at the same time, and each slot works through the keys in
+// blocks of 64 with two score buffers in tensor memory and two probability
+// tiles in shared memory, so that the tensor core, the exponential unit and the
+// barrier round trips overlap.  The stream of blocks runs on across unit
+// boundaries: the first score product of the next unit is issued while the
+// last blocks of the current one are still being exponentiated.
+//
+//   warp 8, one lane : TMA producer (K, V once per unit; Q once per slot).
+//   warps 9, 10      : score issuers, one lane each, one per slot: for block g of
+//                      64 keys S = Q K_g^T (128 x 64 x 64) into one of the slot's
+//                      two score buffers, as soon as that buffer is free; they
+//                      run ahead of the softmax by up to two blocks, also across
+//                      unit boundaries.
+//   warps 11, 12     : output issuers, one lane each, one per slot: when the
+//                      slot's softmax warps have published P_g,
+//                      O += P_g V_g (128 x 64 x 64) into the slot's 64 output
+//                      columns.  (A single issuing thread for all four streams
+//                      was the bottleneck: the per-product bookkeeping of one
+//                      thread cost more than the products themselves.)
+//   warps 0-3, 4-7   : softmax of slot 0 / slot 1, one thread per query row.
+//                      The row keeps a reference exponent m (the maximum of its
+//                      first block).  For each block it forms
+//                      p = 2^(s * log2(e) / 8 - m) from the scores in tensor
+//                      memory, adds them to the fp32 row sum l and writes P as
+//                      bf16 into the swizzled shared-memory tile the MMA reads
+//                      as its A operand.  While doing so it tracks the largest
+//                      exponent of the block; only if that exceeds 16 (p would
+//                      still be far from overflow) is m raised, O and l rescaled
+//                      by 2^(m_old - m_new) through a tensor-memory load / store
+//                      round trip, and the block redone.  O / l is therefore the
+//                      exact softmax for any finite input, and on ordinary
+//                      inputs every score is read once.  Finally the thread
+//                      reads its O row, divides by l and stores 64 bf16 values
+//                      (128 contiguous bytes) to Ctx.
+// Keys beyond the sequence length are zero-filled by TMA and masked out; query
+// rows beyond it are computed and discarded.
 // Every mbarrier wait is bounded (see mbar_wait): on expiry a code is recorded
 // in the device status word, all roles drain, tensor memory is freed and the
 // kernel returns.
-#include "pd_common.cuh"
-#include "sm100_ptx.cuh"
+#include "gemm_common.cuh"
 
 namespace pd {
 namespace {
@@ -42,28 +55,33 @@ namespace {
 using namespace sm100;
 
 constexpr int kD = 64;            // head dimension
-constexpr int kBlockQ = 128;      // queries per block = TMEM lanes
-constexpr int kBlockK = 128;      // keys per score block
-constexpr int kMaxKeys = 512;     // TMEM columns
-constexpr int kQBlocksPerUnit = 2;
-constexpr int kThreads = 320;
-constexpr int kSoftmaxThreads = 256;
-constexpr int kHalfThreads = 128;
-constexpr int kProducerWarp = 8, kMmaWarp = 9;
+constexpr int kBlockQ = 128;      // queries per slot = TMEM lanes
+constexpr int kBlockK = 64;       // keys per score block
+constexpr int kMaxKeys = 512;
+constexpr int kSlots = 2;         // query blocks in flight
+constexpr int kThreads = 416;
+constexpr int kSlotThreads = 128;
+constexpr int kProducerWarp = 8, kScoreWarp0 = 9, kOutputWarp0 = 11, kAllocWarp = 9;
 
 constexpr int kSmemK = kMaxKeys * kD * 2;        // 64 KiB
 constexpr int kSmemV = kMaxKeys * kD * 2;        // 64 KiB
-constexpr int kSmemQ = kBlockQ * kD * 2;         // 16 KiB
-constexpr int kSmemP = kBlockQ * kBlockK * 2;    // 32 KiB per buffer, two buffers
-constexpr int kSmemCtrl = 4096;
-constexpr int kSmemBytes = kSmemK + kSmemV + kSmemQ + 2 * kSmemP + kSmemCtrl + 1024 /*alignment slack*/;
+constexpr int kSmemQ = kBlockQ * kD * 2;         // 16 KiB per slot
+constexpr int kSmemP = kBlockQ * kBlockK * 2;    // 16 KiB per probability tile, two per slot
+constexpr int kSmemCtrl = 1024;
+constexpr int kSmemBytes = kSmemK + kSmemV + kSlots * (kSmemQ + 2 * kSmemP) + kSmemCtrl + 1024 /*alignment slack*/;
+
+// tensor-memory columns: score buffer b of slot s at 128*s + 64*b, output accumulator of slot s at 256 + 64*s
+constexpr uint32_t kTmemS = 0, kTmemO = 256, kTmemCols = 512;
+
+constexpr float kScale = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
+constexpr float kRescaleThreshold = 16.0f;               // largest exponent of 2 tolerated before m is raised
 
 struct AttnParams {
   __nv_bfloat16* ctx;  // [batch*seq, hidden]
   int* status;
   int batch, seq, heads, hidden;
   int q_blocks;   // ceil(seq / 128)
-  int k_blocks;   // ceil(seq / 128)
+  int k_blocks;   // ceil(seq / 64)
   int units_per_head, num_units;
 };
 
@@ -86,35 +104,42 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t sK = smem_base, sV = sK + kSmemK, sQ = sV + kSmemV, sP = sQ + kSmemQ;
-  const uint32_t bar_base = sP + 2 * kSmemP;
-  // barriers (8 bytes each)
+  const uint32_t sK = smem_base, sV = sK + kSmemK, sQ = sV + kSmemV, sP = sQ + kSlots * kSmemQ;
+  const uint32_t bar_base = sP + kSlots * 2 * kSmemP;
+  // barriers (8 bytes each); [s] = slot, [s][b] = slot and buffer
   const uint32_t k_full = bar_base + 0, v_full = bar_base + 8, k_empty = bar_base + 16, v_empty = bar_base + 24;
-  const uint32_t q_full = bar_base + 32, q_empty = bar_base + 40, s_full = bar_base + 48, s_empty = bar_base + 56;
-  const uint32_t o_full = bar_base + 64, drain_bar = bar_base + 72;
-  auto p_full = [&](int i) { return bar_base + 80u + 8u * i; };
-  auto p_empty = [&](int i) { return bar_base + 96u + 8u * i; };
-  const uint32_t max_bar = bar_base + 112, sum_bar = bar_base + 120;
-  uint8_t* ctrl = smem_gen + (bar_base - smem_base) + 128;
+  auto q_full = [&](int s) { return bar_base + 40u + 8u * s; };
+  auto q_empty = [&](int s) { return bar_base + 56u + 8u * s; };
+  auto o_full = [&](int s) { return bar_base + 72u + 8u * s; };
+  auto o_empty = [&](int s) { return bar_base + 88u + 8u * s; };
+  auto s_full = [&](int s, int b) { return bar_base + 104u + 8u * (2 * s + b); };
+  auto s_empty = [&](int s, int b) { return bar_base + 136u + 8u * (2 * s + b); };
+  auto p_full = [&](int s, int b) { return bar_base + 168u + 8u * (2 * s + b); };
+  auto p_empty = [&](int s, int b) { return bar_base + 200u + 8u * (2 * s + b); };
+  const uint32_t drain_bar = bar_base + 232;  // four of them, one per MMA-issuing warp
+  uint8_t* ctrl = smem_gen + (bar_base - smem_base) + 512;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 4);
-  float* xmax = reinterpret_cast<float*>(ctrl + 1024);  // [2][128] row maxima of the two halves
-  float* xsum = reinterpret_cast<float*>(ctrl + 2048);  // [2][128] partial row sums
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    mbar_init(k_full, 1); mbar_init(v_full, 1); mbar_init(k_empty, 1); mbar_init(v_empty, 1);
-    mbar_init(q_full, 1); mbar_init(q_empty, 1); mbar_init(s_full, 1); mbar_init(s_empty, kSoftmaxThreads);
-    mbar_init(o_full, 1); mbar_init(drain_bar, 1);
-    mbar_init(max_bar, kSoftmaxThreads); mbar_init(sum_bar, kSoftmaxThreads);
-    for (int i = 0; i < 2; ++i) { mbar_init(p_full(i), kHalfThreads); mbar_init(p_empty(i), 1); }
+    mbar_init(k_full, 1); mbar_init(v_full, 1); mbar_init(k_empty, kSlots); mbar_init(v_empty, kSlots);
+    for (int i = 0; i < 4; ++i) mbar_init(drain_bar + 8u * i, 1);
+    for (int s = 0; s < kSlots; ++s) {
+      mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1);
+      mbar_init(o_full(s), 1); mbar_init(o_empty(s), kSlotThreads);
+      for (int b = 0; b < 2; ++b) {
+        mbar_init(s_full(s, b), 1); mbar_init(s_empty(s, b), kSlotThreads);
+        mbar_init(p_full(s, b), kSlotThreads); mbar_init(p_empty(s, b), 1);
+      }
+    }
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
   }
-  if (warp == kMmaWarp) {
-    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), 512);
+  if (warp == kAllocWarp) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
     tmem_relinquish_alloc_permit();
   }
   tcgen05_fence_before_sync();
@@ -122,221 +147,268 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  // Work decomposition shared by all roles.
-  auto unit_coords = [&](int unit, int& b, int& h, int& qb0, int& nqb) {
+  // Work decomposition shared by all roles: unit -> (batch, head, first query block, active slots).
+  auto unit_coords = [&](int unit, int& b, int& h, int& qb0, int& nslots) {
     const int per_bh = p.units_per_head;
     const int bh = unit / per_bh;
     b = bh / p.heads;
     h = bh % p.heads;
-    qb0 = (unit % per_bh) * kQBlocksPerUnit;
-    nqb = min(kQBlocksPerUnit, p.q_blocks - qb0);
+    qb0 = (unit % per_bh) * kSlots;
+    nslots = min(kSlots, p.q_blocks - qb0);
   };
+  const int G = p.k_blocks;
 
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------- TMA producer
     if (lane == 0) {
       prefetch_tensormap(&tmap_q); prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v);
-      uint32_t n_unit = 0, n_q = 0;
+      uint32_t n_unit = 0, n_q0 = 0, n_q1 = 0;
       bool ok = true;
       for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x, ++n_unit) {
-        int b, h, qb0, nqb;
-        unit_coords(unit, b, h, qb0, nqb);
-        const uint32_t uph = n_unit & 1u;
-        if (!mbar_wait(k_empty, uph ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
+        int b, h, qb0, nslots;
+        unit_coords(unit, b, h, qb0, nslots);
+        if (!mbar_wait(k_empty, (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
         mbar_arrive_expect_tx(k_full, kSmemK);
         tma_load_4d(sK, &tmap_k, k_full, 0, 0, h, b);
         tma_load_4d(sK + kSmemK / 2, &tmap_k, k_full, 0, 256, h, b);
-        // the first Q of the unit goes out before V: the score product needs only Q and K
-        for (int i = 0; i < nqb && ok; ++i, ++n_q) {
-          if (!mbar_wait(q_empty, (n_q & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
-          mbar_arrive_expect_tx(q_full, kSmemQ);
-          tma_load_4d(sQ, &tmap_q, q_full, 0, (qb0 + i) * kBlockQ, h, b);
-          if (i == 0) {
-            if (!mbar_wait(v_empty, uph ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
-            mbar_arrive_expect_tx(v_full, kSmemV);
-            tma_load_4d(sV, &tmap_v, v_full, 0, 0, h, b);
-            tma_load_4d(sV + kSmemV / 2, &tmap_v, v_full, 0, 256, h, b);
-          }
+        for (int s = 0; s < nslots && ok; ++s) {
+          const uint32_t nq = s ? n_q1 : n_q0;
+          if (!mbar_wait(q_empty(s), (nq & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
+          if (s) ++n_q1; else ++n_q0;
+          mbar_arrive_expect_tx(q_full(s), kSmemQ);
+          tma_load_4d(sQ + s * kSmemQ, &tmap_q, q_full(s), 0, (qb0 + s) * kBlockQ, h, b);
         }
+        if (!ok) break;
+        if (!mbar_wait(v_empty, (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
+        mbar_arrive_expect_tx(v_full, kSmemV);
+        tma_load_4d(sV, &tmap_v, v_full, 0, 0, h, b);
+        tma_load_4d(sV + kSmemV / 2, &tmap_v, v_full, 0, 256, h, b);
       }
-      if (!ok) {
-        // leave no copy in flight: give the last armed barriers a short time to complete
+      if (!ok && n_unit > 0) {
+        // leave no copy in flight: give the barriers armed last a short time to complete
         volatile int never = 0;
-        if (n_unit > 0 || n_q > 0) {
-          mbar_wait(k_full, (n_unit & 1u), &never, nullptr, 0, 20000000ull);
-          mbar_wait(q_full, ((n_q - 1u) & 1u), &never, nullptr, 0, 20000000ull);
-        }
+        mbar_wait(k_full, (n_unit - 1u) & 1u, &never, nullptr, 0, 20000000ull);
+        mbar_wait(v_full, (n_unit - 1u) & 1u, &never, nullptr, 0, 20000000ull);
       }
     }
-  } else if (warp == kMmaWarp) {
-    // --------------------------------------------------------------- MMA issuer
+  } else if (warp == kScoreWarp0 || warp == kScoreWarp0 + 1) {
+    // ------------------------------------------- score-product issuer of one slot
     if (lane == 0) {
+      const int s = warp - kScoreWarp0;
       constexpr uint32_t idesc_s = make_idesc_bf16(kBlockQ, kBlockK, false, false);  // Q K^T: both K-major
-      constexpr uint32_t idesc_o = make_idesc_bf16(kBlockQ, kD, false, true);        // P V: V is MN-major
-      uint32_t n_unit = 0, n_q = 0, n_use0 = 0, n_use1 = 0;  // fills of each half's P tile consumed so far
+      const uint64_t q_desc = make_smem_desc(sQ + s * kSmemQ, 0, 1024);
+      const uint64_t k_desc = make_smem_desc(sK, 0, 1024);
+      const uint32_t d_tmem = tmem_base + kTmemS + s * 128;
+      uint32_t t = 0, n_q = 0, n_unit = 0;
       bool ok = true;
       for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x, ++n_unit) {
-        int b, h, qb0, nqb;
-        unit_coords(unit, b, h, qb0, nqb);
-        const uint32_t uph = n_unit & 1u;
-        if (!mbar_wait(k_full, uph, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-        for (int i = 0; i < nqb && ok; ++i, ++n_q) {
-          const uint32_t qph = n_q & 1u;
-          if (!mbar_wait(q_full, qph, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-          if (!mbar_wait(s_empty, qph ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-          tcgen05_fence_after_sync();
-          for (int j = 0; j < p.k_blocks; ++j) {
-#pragma unroll
-            for (int ks = 0; ks < kD / 16; ++ks) {
-              const uint64_t a_desc = make_smem_desc(sQ + ks * 32, 0, 1024);
-              const uint64_t b_desc = make_smem_desc(sK + j * (kBlockK * 128) + ks * 32, 0, 1024);
-              mma_bf16_ss(tmem_base + j * kBlockK, a_desc, b_desc, idesc_s, ks != 0 ? 1u : 0u);
-            }
-          }
-          mma_commit(s_full);
-          mma_commit(q_empty);
-          if (i == nqb - 1) mma_commit(k_empty);
-          if (i == 0 && !mbar_wait(v_full, uph, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-          for (int j = 0; j < p.k_blocks && ok; ++j) {
-            const int buf = j & 1;  // key block j is produced by softmax half j % 2 into its own tile
-            const uint32_t use = buf ? n_use1 : n_use0;
-            if (!mbar_wait(p_full(buf), use & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-            if (buf) ++n_use1; else ++n_use0;
+        int b, h, qb0, nslots;
+        unit_coords(unit, b, h, qb0, nslots);
+        if (!mbar_wait(k_full, n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+        if (s < nslots) {
+          if (!mbar_wait(q_full(s), n_q & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+          ++n_q;
+          for (int g = 0; g < G; ++g, ++t) {
+            const uint32_t buf = t & 1u;
+            if (!mbar_wait(s_empty(s, buf), ((t >> 1) & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
             tcgen05_fence_after_sync();
+            const uint64_t kg = k_desc + (uint64_t)(g * ((kBlockK * 128) >> 4));
 #pragma unroll
-            for (int ks = 0; ks < kBlockK / 16; ++ks) {
-              const uint64_t a_desc = make_smem_desc(sP + buf * kSmemP + (ks >> 2) * (kBlockQ * 128) + (ks & 3) * 32, 0, 1024);
-              const uint64_t b_desc = make_smem_desc(sV + (j * kBlockK + ks * 16) * 128, 0, 1024);
-              mma_bf16_ss(tmem_base, a_desc, b_desc, idesc_o, (j | ks) != 0 ? 1u : 0u);
-            }
-            mma_commit(p_empty(buf));
+            for (int ks = 0; ks < kD / 16; ++ks)
+              mma_bf16_ss(d_tmem + buf * kBlockK, q_desc + 2 * ks, kg + 2 * ks, idesc_s, ks != 0 ? 1u : 0u);
+            mma_commit(s_full(s, buf));
           }
           if (!ok) break;
-          mma_commit(o_full);
-          if (i == nqb - 1) mma_commit(v_empty);
+          mma_commit(q_empty(s));
         }
+        mma_commit(k_empty);  // both score issuers arrive, whether or not their slot is in use
       }
       if (!ok) {
-        mma_commit(drain_bar);
+        mma_commit(drain_bar + 16u + 8u * s);
         volatile int never = 0;
-        mbar_wait(drain_bar, 0, &never, nullptr, 0, 20000000ull);
+        mbar_wait(drain_bar + 16u + 8u * s, 0, &never, nullptr, 0, 20000000ull);
+      }
+    }
+  } else if (warp == kOutputWarp0 || warp == kOutputWarp0 + 1) {
+    // --------------------------------------------- P V product issuer of one slot
+    if (lane == 0) {
+      const int s = warp - kOutputWarp0;
+      constexpr uint32_t idesc_o = make_idesc_bf16(kBlockQ, kD, false, true);  // V is MN-major
+      const uint64_t p_desc = make_smem_desc(sP + 2 * s * kSmemP, 0, 1024);
+      const uint64_t v_desc = make_smem_desc(sV, 0, 1024);
+      const uint32_t d_tmem = tmem_base + kTmemO + s * kD;
+      uint32_t t = 0, n_us = 0, n_unit = 0;
+      bool ok = true;
+      for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x, ++n_unit) {
+        int b, h, qb0, nslots;
+        unit_coords(unit, b, h, qb0, nslots);
+        if (!mbar_wait(v_full, n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+        if (s < nslots) {
+          // the previous unit's output of this slot must have been read before it is overwritten
+          if (!mbar_wait(o_empty(s), (n_us & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+          for (int g = 0; g < G; ++g, ++t) {
+            const uint32_t buf = t & 1u;
+            if (!mbar_wait(p_full(s, buf), (t >> 1) & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+            tcgen05_fence_after_sync();
+            const uint64_t pg = p_desc + (uint64_t)(buf * (kSmemP >> 4));
+            const uint64_t vg = v_desc + (uint64_t)(g * ((kBlockK * 128) >> 4));
+#pragma unroll
+            for (int ks = 0; ks < kBlockK / 16; ++ks)
+              mma_bf16_ss(d_tmem, pg + 2 * ks, vg + ks * ((16 * 128) >> 4), idesc_o, (g | ks) != 0 ? 1u : 0u);
+            mma_commit(p_empty(s, buf));
+          }
+          if (!ok) break;
+          mma_commit(o_full(s));
+          ++n_us;
+        }
+        mma_commit(v_empty);  // both output issuers arrive
+      }
+      if (!ok) {
+        mma_commit(drain_bar + 8u * s);
+        volatile int never = 0;
+        mbar_wait(drain_bar + 8u * s, 0, &never, nullptr, 0, 20000000ull);
       }
     }
   } else {
     // ------------------------------------------------------------------ softmax
-    const int quarter = warp & 3, half = warp >> 2;
+    const int slot = warp >> 2, quarter = warp & 3;
     const int row = quarter * 32 + lane;  // query row within the block = TMEM lane
-    const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t t_o = t_lane + kTmemO + slot * kD;
     const uint32_t sw = (uint32_t)(lane & 7);
-    const float kScale = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
-    const uint32_t p_row = sP + half * kSmemP + (uint32_t)row * 128u;
-    uint32_t n_q = 0, n_use = 0;  // n_use: how often this half has filled its P tile
+    uint32_t t = 0, n_us = 0;  // score blocks and units this slot has processed
     bool ok = true;
     for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x) {
-      int b, h, qb0, nqb;
-      unit_coords(unit, b, h, qb0, nqb);
-      for (int i = 0; i < nqb && ok; ++i, ++n_q) {
-        const uint32_t qph = n_q & 1u;
-        if (!mbar_wait(s_full, qph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+      int b, h, qb0, nslots;
+      unit_coords(unit, b, h, qb0, nslots);
+      if (slot >= nslots) continue;
+      float mk = 0.f, l = 0.f;  // reference exponent (already scaled by log2(e)/8) and row sum
+      for (int g = 0; g < G && ok; ++g, ++t) {
+        const int buf = t & 1u;
+        const uint32_t use_ph = (t >> 1) & 1u;
+        const uint32_t t_s = t_lane + kTmemS + slot * 128 + buf * kBlockK;
+        const uint32_t p_row = sP + (2 * slot + buf) * kSmemP + (uint32_t)row * 128u;
+        const int key0 = g * kBlockK;
+        if (!mbar_wait(s_full(slot, buf), use_ph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
         tcgen05_fence_after_sync();
-        // pass 1: maximum over this half's key blocks (j = half, half + 2), loads one chunk ahead
-        float m = -INFINITY;
-        {
-          const int n_chunks = ((p.k_blocks - half + 1) >> 1) * (kBlockK / 32);  // 4 chunks per block
-          auto col_of = [&](int c) { return ((c >> 2) * 2 + half) * kBlockK + (c & 3) * 32; };
-          uint32_t r[2][32];
-          if (n_chunks > 0) tmem_ld_32x32b_x32(t_row + col_of(0), r[0]);
-#pragma unroll 1
-          for (int c = 0; c < n_chunks; c += 2) {
-#pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              if (c + u >= n_chunks) break;
-              tmem_ld_wait();
-              if (c + u + 1 < n_chunks) tmem_ld_32x32b_x32(t_row + col_of(c + u + 1), r[u ^ 1]);
-              const int c0 = col_of(c + u);
-              if (c0 + 32 <= p.seq) {
-#pragma unroll
-                for (int t = 0; t < 32; ++t) m = fmaxf(m, __uint_as_float(r[u][t]));
-              } else {
-#pragma unroll
-                for (int t = 0; t < 32; ++t)
-                  if (c0 + t < p.seq) m = fmaxf(m, __uint_as_float(r[u][t]));
-              }
-            }
-          }
-        }
-        xmax[half * kBlockQ + row] = m;
-        mbar_arrive(max_bar);
-        if (!mbar_wait(max_bar, qph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
-        m = fmaxf(xmax[row], xmax[kBlockQ + row]);
-        const float mk = m * kScale;
-        // pass 2: probabilities of this half's key blocks
-        float sum = 0.f;
-        for (int j = half; j < p.k_blocks && ok; j += 2, ++n_use) {
-          if (!mbar_wait(p_empty(half), (n_use & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
-          uint32_t r[2][32];
-          tmem_ld_32x32b_x32(t_row + j * kBlockK, r[0]);
+        if (g == 0) {
+          // the first block fixes the reference: its maximum
+          float bm = -INFINITY;
 #pragma unroll
           for (int cc = 0; cc < kBlockK / 32; ++cc) {
-            const int c = cc * 32;
-            const int c0 = j * kBlockK + c;
+            uint32_t r[32];
+            tmem_ld_32x32b_x32(t_s + cc * 32, r);
             tmem_ld_wait();
-            if (cc + 1 < kBlockK / 32) tmem_ld_32x32b_x32(t_row + c0 + 32, r[(cc & 1) ^ 1]);
+            const int c0 = key0 + cc * 32;
+            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c0 + i < p.seq) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(r[i]));
+            bm = fmaxf(bm, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+          }
+          mk = bm * kScale;
+        }
+        // P_{g-2} V_{g-2} read the tile rewritten below: it must have completed
+        if (!mbar_wait(p_empty(slot, buf), use_ph ^ 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+        // exponentials of the block against reference `ref`: writes P, returns the row's partial sum and
+        // the largest exponent met
+        auto exp_block = [&](float ref, float& part_out, float& amax_out) {
+          float part = 0.f;
+          float a4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          uint32_t r[2][32];
+          tmem_ld_32x32b_x32(t_s, r[0]);
+#pragma unroll
+          for (int cc = 0; cc < kBlockK / 32; ++cc) {
+            tmem_ld_wait();
+            if (cc + 1 < kBlockK / 32) tmem_ld_32x32b_x32(t_s + (cc + 1) * 32, r[(cc & 1) ^ 1]);
             const uint32_t(&rr)[32] = r[cc & 1];
+            const int c0 = key0 + cc * 32;
             float e[32];
             if (c0 + 32 <= p.seq) {
 #pragma unroll
-              for (int t = 0; t < 32; ++t) e[t] = ex2_approx(fmaf(__uint_as_float(rr[t]), kScale, -mk));
+              for (int i = 0; i < 32; ++i) {
+                const float a = fmaf(__uint_as_float(rr[i]), kScale, -ref);
+                a4[i & 3] = fmaxf(a4[i & 3], a);
+                e[i] = ex2_approx(a);
+              }
             } else {
 #pragma unroll
-              for (int t = 0; t < 32; ++t)
-                e[t] = (c0 + t < p.seq) ? ex2_approx(fmaf(__uint_as_float(rr[t]), kScale, -mk)) : 0.f;
+              for (int i = 0; i < 32; ++i) {
+                const float a = fmaf(__uint_as_float(rr[i]), kScale, -ref);
+                const bool valid = c0 + i < p.seq;
+                if (valid) a4[i & 3] = fmaxf(a4[i & 3], a);
+                e[i] = valid ? ex2_approx(a) : 0.f;
+              }
             }
-            float part = 0.f;
 #pragma unroll
-            for (int t = 0; t < 32; t += 4) part += (e[t] + e[t + 1]) + (e[t + 2] + e[t + 3]);
-            sum += part;
-            // keys c .. c+31 of the block: 16-byte units (c%64)/8 .. +3 of sub-tile c/64
-            const uint32_t sub = p_row + (uint32_t)(c >> 6) * (kBlockQ * 128u);
-            const uint32_t u0 = (uint32_t)((c & 63) >> 3);
+            for (int i = 0; i < 32; i += 4) part += (e[i] + e[i + 1]) + (e[i + 2] + e[i + 3]);
+            // keys 32*cc .. 32*cc+31 of the block: 16-byte units 4*cc .. 4*cc+3 of the row
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-              st_shared_v4(sub + (((u0 + u) ^ sw) << 4),
+              st_shared_v4(p_row + (((uint32_t)(4 * cc + u) ^ sw) << 4),
                            make_uint4(pack_bf16x2(e[8 * u], e[8 * u + 1]), pack_bf16x2(e[8 * u + 2], e[8 * u + 3]),
                                       pack_bf16x2(e[8 * u + 4], e[8 * u + 5]), pack_bf16x2(e[8 * u + 6], e[8 * u + 7])));
           }
-          fence_proxy_async_smem();
-          mbar_arrive(p_full(half));
-        }
-        if (!ok) break;
-        xsum[half * kBlockQ + row] = sum;
-        mbar_arrive(sum_bar);
-        if (!mbar_wait(sum_bar, qph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
-        const float inv = 1.0f / (xsum[row] + xsum[kBlockQ + row]);
-        // output: this half's 32 columns of O / sum -> bf16 -> Ctx
-        if (!mbar_wait(o_full, qph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
-        tcgen05_fence_after_sync();
-        const int q = (qb0 + i) * kBlockQ + row;
-        __nv_bfloat16* out = p.ctx + ((int64_t)b * p.seq + q) * p.hidden + h * kD + half * 32;
-        {
-          uint32_t r[32];
-          tmem_ld_32x32b_x32(t_row + half * 32, r);
-          tmem_ld_wait();
-          if (q < p.seq) {
+          part_out = part;
+          amax_out = fmaxf(fmaxf(a4[0], a4[1]), fmaxf(a4[2], a4[3]));
+        };
+        float part, amax;
+        exp_block(mk, part, amax);
+        const bool raise = amax > kRescaleThreshold;
+        if (__any_sync(0xffffffffu, raise)) {
+          // rare: this block towers over the reference.  Raise the reference of the rows concerned, rescale
+          // what they have accumulated, and redo the block.  Every earlier P V product of the slot has to
+          // be complete before O is touched: the latest one is the other tile's (there is one: g >= 1).
+          if (!mbar_wait(p_empty(slot, buf ^ 1), ((t - 1u) >> 1) & 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+          tcgen05_fence_after_sync();
+          const float alpha = raise ? ex2_approx(-amax) : 1.0f;
+          if (raise) mk += amax;
+          l *= alpha;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              uint4 w;
-              w.x = pack_bf16x2(__uint_as_float(r[8 * u]) * inv, __uint_as_float(r[8 * u + 1]) * inv);
-              w.y = pack_bf16x2(__uint_as_float(r[8 * u + 2]) * inv, __uint_as_float(r[8 * u + 3]) * inv);
-              w.z = pack_bf16x2(__uint_as_float(r[8 * u + 4]) * inv, __uint_as_float(r[8 * u + 5]) * inv);
-              w.w = pack_bf16x2(__uint_as_float(r[8 * u + 6]) * inv, __uint_as_float(r[8 * u + 7]) * inv);
-              *reinterpret_cast<uint4*>(out + 8 * u) = w;
-            }
+          for (int c0 = 0; c0 < kD; c0 += 32) {
+            uint32_t o[32];
+            tmem_ld_32x32b_x32(t_o + c0, o);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            tmem_st_32x32b_x32(t_o + c0, o);
+          }
+          tmem_st_wait();
+          exp_block(mk, part, amax);
+        }
+        l += part;
+        fence_proxy_async_smem();
+        tcgen05_fence_before_sync();
+        mbar_arrive(p_full(slot, buf));
+        mbar_arrive(s_empty(slot, buf));
+      }
+      if (!ok) break;
+      // ---- output: O / l -> bf16 -> Ctx
+      if (!mbar_wait(o_full(slot), n_us & 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+      ++n_us;
+      tcgen05_fence_after_sync();
+      const float inv = 1.0f / l;
+      const int q = (qb0 + slot) * kBlockQ + row;
+      __nv_bfloat16* out = p.ctx + ((int64_t)b * p.seq + q) * p.hidden + h * kD;
+#pragma unroll
+      for (int c0 = 0; c0 < kD; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(t_o + c0, r);
+        tmem_ld_wait();
+        if (q < p.seq) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(r[8 * u]) * inv, __uint_as_float(r[8 * u + 1]) * inv);
+            w.y = pack_bf16x2(__uint_as_float(r[8 * u + 2]) * inv, __uint_as_float(r[8 * u + 3]) * inv);
+            w.z = pack_bf16x2(__uint_as_float(r[8 * u + 4]) * inv, __uint_as_float(r[8 * u + 5]) * inv);
+            w.w = pack_bf16x2(__uint_as_float(r[8 * u + 6]) * inv, __uint_as_float(r[8 * u + 7]) * inv);
+            *reinterpret_cast<uint4*>(out + c0 + 8 * u) = w;
           }
         }
-        tcgen05_fence_before_sync();
-        mbar_arrive(s_empty);
       }
+      tcgen05_fence_before_sync();
+      mbar_arrive(o_empty(slot));
     }
   }
 
@@ -344,32 +416,16 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   __syncwarp();
   tcgen05_fence_before_sync();
   __syncthreads();
-  if (warp == kMmaWarp) {
+  if (warp == kAllocWarp) {
     tcgen05_fence_after_sync();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc(tmem_base, kTmemCols);
   }
-}
-
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = [] {
-    void* f = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      f = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(f);
-  }();
-  return fn;
 }
 
 // One of Q, K, V inside qkv[batch*seq, 3*hidden]: dims {64, seq, heads, batch}.
 bool make_head_map(CUtensorMap* map, const __nv_bfloat16* base, int64_t seq, int64_t heads, int64_t batch,
                    int64_t hidden, int box_rows) {
-  EncodeTiledFn fn = encode_tiled_fn();
+  gemm::EncodeTiledFn fn = gemm::encode_tiled_fn();
   if (!fn) return false;
   const cuuint64_t dims[4] = {(cuuint64_t)kD, (cuuint64_t)seq, (cuuint64_t)heads, (cuuint64_t)batch};
   const cuuint64_t strides[3] = {(cuuint64_t)(3 * hidden) * 2, (cuuint64_t)kD * 2, (cuuint64_t)(seq * 3 * hidden) * 2};
@@ -398,8 +454,8 @@ pd_status launch_fused_attention(const __nv_bfloat16* qkv, __nv_bfloat16* ctx, i
   if (!p.status) return PD_ERR_CUDA;
   p.batch = (int)batch; p.seq = (int)seq; p.heads = (int)heads; p.hidden = (int)hidden;
   p.q_blocks = (int)((seq + kBlockQ - 1) / kBlockQ);
-  p.k_blocks = (int)((seq + kBlockK - 1) / kBlockK);
-  p.units_per_head = (p.q_blocks + kQBlocksPerUnit - 1) / kQBlocksPerUnit;
+  p.k_blocks = (int)((seq + kBlockK - 1) / kBlockK);  // blocks of 64 keys
+  p.units_per_head = (p.q_blocks + kSlots - 1) / kSlots;
   const int64_t units = batch * heads * p.units_per_head;
   if (units > 0x7fffffff) return PD_ERR_BAD_SHAPE;
   p.num_units = (int)units;
