@@ -5,7 +5,7 @@
 // on the packed projection qkv[tokens, 3*hidden] = [Q | K | V].  Scores and
 // probabilities never leave the SM.
 //
-// One persistent CTA of 416 threads per SM walks over work units of (batch,
+// One persistent CTA of 352 threads per SM walks over work units of (batch,
 // head, pair of 128-query blocks).  K and V of the head (up to 512 x 64 each)
 // are resident in shared memory for the unit; the two query blocks ("slots")
 // are in flight at the same time, and each slot works through the keys in
@@ -16,12 +16,12 @@
 // last blocks of the current one are still being exponentiated.
 //
 //   warp 8, one lane : TMA producer (K, V once per unit; Q once per slot).
-//   warps 9, 10      : score issuers, one lane each, one per slot: for block g of
+//   warp 9, lanes 0-1: score issuers, one thread per slot: for block g of
 //                      64 keys S = Q K_g^T (128 x 64 x 64) into one of the slot's
 //                      two score buffers, as soon as that buffer is free; they
 //                      run ahead of the softmax by up to two blocks, also across
 //                      unit boundaries.
-//   warps 11, 12     : output issuers, one lane each, one per slot: when the
+//   warp 10, lanes 0-1: output issuers, one thread per slot: when the
 //                      slot's softmax warps have published P_g,
 //                      O += P_g V_g (128 x 64 x 64) into the slot's 64 output
 //                      columns.  (A single issuing thread for all four streams
@@ -40,8 +40,9 @@
 //                      round trip, and the block redone.  O / l is therefore the
 //                      exact softmax for any finite input, and on ordinary
 //                      inputs every score is read once.  Finally the thread
-//                      reads its O row, divides by l and stores 64 bf16 values
-//                      (128 contiguous bytes) to Ctx.
+//                      reads its O row, divides by l and stages 64 bf16 values
+//                      in the (by then idle) probability tile, from where each
+//                      warp's 32 rows go to Ctx with one TMA store.
 // Keys beyond the sequence length are zero-filled by TMA and masked out; query
 // rows beyond it are computed and discarded.
 // Every mbarrier wait is bounded (see mbar_wait): on expiry a code is recorded
@@ -59,9 +60,9 @@ constexpr int kBlockQ = 128;      // queries per slot = TMEM lanes
 constexpr int kBlockK = 64;       // keys per score block
 constexpr int kMaxKeys = 512;
 constexpr int kSlots = 2;         // query blocks in flight
-constexpr int kThreads = 416;
+constexpr int kThreads = 352;
 constexpr int kSlotThreads = 128;
-constexpr int kProducerWarp = 8, kScoreWarp0 = 9, kOutputWarp0 = 11, kAllocWarp = 9;
+constexpr int kProducerWarp = 8, kScoreWarp = 9, kOutputWarp = 10, kAllocWarp = 9;
 
 constexpr int kSmemK = kMaxKeys * kD * 2;        // 64 KiB
 constexpr int kSmemV = kMaxKeys * kD * 2;        // 64 KiB
@@ -100,7 +101,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 __global__ void __launch_bounds__(kThreads, 1)
 attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                             const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
+                             const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+                             const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -191,10 +193,10 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         mbar_wait(v_full, (n_unit - 1u) & 1u, &never, nullptr, 0, 20000000ull);
       }
     }
-  } else if (warp == kScoreWarp0 || warp == kScoreWarp0 + 1) {
-    // ------------------------------------------- score-product issuer of one slot
-    if (lane == 0) {
-      const int s = warp - kScoreWarp0;
+  } else if (warp == kScoreWarp) {
+    // ---------------------- score-product issuers: lane 0 for slot 0, lane 1 for slot 1
+    if (lane < kSlots) {
+      const int s = lane;
       constexpr uint32_t idesc_s = make_idesc_bf16(kBlockQ, kBlockK, false, false);  // Q K^T: both K-major
       const uint64_t q_desc = make_smem_desc(sQ + s * kSmemQ, 0, 1024);
       const uint64_t k_desc = make_smem_desc(sK, 0, 1024);
@@ -229,10 +231,10 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         mbar_wait(drain_bar + 16u + 8u * s, 0, &never, nullptr, 0, 20000000ull);
       }
     }
-  } else if (warp == kOutputWarp0 || warp == kOutputWarp0 + 1) {
-    // --------------------------------------------- P V product issuer of one slot
-    if (lane == 0) {
-      const int s = warp - kOutputWarp0;
+  } else if (warp == kOutputWarp) {
+    // ------------------------ P V product issuers: lane 0 for slot 0, lane 1 for slot 1
+    if (lane < kSlots) {
+      const int s = lane;
       constexpr uint32_t idesc_o = make_idesc_bf16(kBlockQ, kD, false, true);  // V is MN-major
       const uint64_t p_desc = make_smem_desc(sP + 2 * s * kSmemP, 0, 1024);
       const uint64_t v_desc = make_smem_desc(sV, 0, 1024);
@@ -278,6 +280,7 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
     const uint32_t sw = (uint32_t)(lane & 7);
     uint32_t t = 0, n_us = 0;  // score blocks and units this slot has processed
     bool ok = true;
+    bool store_pending = false;  // this warp's output store may still be reading probability tile 0
     for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x) {
       int b, h, qb0, nslots;
       unit_coords(unit, b, h, qb0, nslots);
@@ -307,6 +310,11 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
             bm = fmaxf(bm, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
           }
           mk = bm * kScale;
+        }
+        if (store_pending && buf == 0) {
+          if (lane == 0) tma_store_wait_read<0>();
+          __syncwarp();
+          store_pending = false;
         }
         // P_{g-2} V_{g-2} read the tile rewritten below: it must have completed
         if (!mbar_wait(p_empty(slot, buf), use_ph ^ 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
@@ -383,33 +391,43 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         mbar_arrive(s_empty(slot, buf));
       }
       if (!ok) break;
-      // ---- output: O / l -> bf16 -> Ctx
+      // ---- output: O / l -> bf16 -> the slot's first probability tile (free by now: every P V product
+      // of the unit has completed) -> one TMA store of 32 rows x 128 bytes per warp; rows beyond the
+      // sequence are clipped by the tensor map
       if (!mbar_wait(o_full(slot), n_us & 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
       ++n_us;
       tcgen05_fence_after_sync();
       const float inv = 1.0f / l;
-      const int q = (qb0 + slot) * kBlockQ + row;
-      __nv_bfloat16* out = p.ctx + ((int64_t)b * p.seq + q) * p.hidden + h * kD;
+      const uint32_t o_row = sP + (2 * slot) * kSmemP + (uint32_t)row * 128u;
 #pragma unroll
       for (int c0 = 0; c0 < kD; c0 += 32) {
         uint32_t r[32];
         tmem_ld_32x32b_x32(t_o + c0, r);
         tmem_ld_wait();
-        if (q < p.seq) {
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            uint4 w;
-            w.x = pack_bf16x2(__uint_as_float(r[8 * u]) * inv, __uint_as_float(r[8 * u + 1]) * inv);
-            w.y = pack_bf16x2(__uint_as_float(r[8 * u + 2]) * inv, __uint_as_float(r[8 * u + 3]) * inv);
-            w.z = pack_bf16x2(__uint_as_float(r[8 * u + 4]) * inv, __uint_as_float(r[8 * u + 5]) * inv);
-            w.w = pack_bf16x2(__uint_as_float(r[8 * u + 6]) * inv, __uint_as_float(r[8 * u + 7]) * inv);
-            *reinterpret_cast<uint4*>(out + c0 + 8 * u) = w;
-          }
+        for (int u = 0; u < 4; ++u) {
+          uint4 w;
+          w.x = pack_bf16x2(__uint_as_float(r[8 * u]) * inv, __uint_as_float(r[8 * u + 1]) * inv);
+          w.y = pack_bf16x2(__uint_as_float(r[8 * u + 2]) * inv, __uint_as_float(r[8 * u + 3]) * inv);
+          w.z = pack_bf16x2(__uint_as_float(r[8 * u + 4]) * inv, __uint_as_float(r[8 * u + 5]) * inv);
+          w.w = pack_bf16x2(__uint_as_float(r[8 * u + 6]) * inv, __uint_as_float(r[8 * u + 7]) * inv);
+          st_shared_v4(o_row + (((uint32_t)(c0 / 8 + u) ^ sw) << 4), w);
         }
       }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_4d(&tmap_o, sP + (2 * slot) * kSmemP + (uint32_t)(quarter * 32) * 128u, 0,
+                     (qb0 + slot) * kBlockQ + quarter * 32, h, b);
+        tma_store_commit();
+      }
+      store_pending = true;
       tcgen05_fence_before_sync();
       mbar_arrive(o_empty(slot));
     }
+    // shared memory must outlive every store that still reads it
+    if (lane == 0) tma_store_wait_all<0>();
+    __syncwarp();
   }
 
   // ------------------------------------------------------------------- teardown
@@ -448,6 +466,9 @@ pd_status launch_fused_attention(const __nv_bfloat16* qkv, __nv_bfloat16* ctx, i
       !make_head_map(&tk, qkv + hidden, seq, heads, batch, hidden, 256) ||
       !make_head_map(&tv, qkv + 2 * hidden, seq, heads, batch, hidden, 256))
     return PD_ERR_UNSUPPORTED;
+  // Ctx[batch*seq, hidden] seen as {64, seq, heads, batch}; written in boxes of 32 rows x 64 columns
+  CUtensorMap to;
+  if (!gemm::make_map(&to, false, ctx, kD, seq, hidden, heads, kD, batch, seq * hidden, kD, 32)) return PD_ERR_UNSUPPORTED;
   AttnParams p{};
   p.ctx = ctx;
   p.status = device_status_ptr();
@@ -467,7 +488,7 @@ pd_status launch_fused_attention(const __nv_bfloat16* qkv, __nv_bfloat16* ctx, i
     attr_set = true;
   }
   const int grid = p.num_units < sm_count() ? p.num_units : sm_count();
-  attention_fwd_tcgen05_kernel<<<grid, kThreads, kSmemBytes, s>>>(tq, tk, tv, p);
+  attention_fwd_tcgen05_kernel<<<grid, kThreads, kSmemBytes, s>>>(tq, tk, tv, to, p);
   return check_launch();
 }
 
