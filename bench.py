@@ -41,7 +41,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel at the FFN-up / configured
 # GEMM shape, from the ncu capture summarised in profiles/gemm_bf16_tcgen05_16384x4096x1024.md.  Set to None
 # whenever that kernel changes until the counters are taken again.
-DOMINANT_KERNEL_DRAM_TRAFFIC_BYTES = 42.008320e6 + 77.843200e6
+DOMINANT_KERNEL_DRAM_TRAFFIC_BYTES = None
 METRIC = "achieved HBM GB/s (row ops) and bf16 TFLOP/s (GEMM, layer) as % of roofline"
 
 
@@ -160,15 +160,40 @@ def run_reference(args):
 # GPU arm
 # ----------------------------------------------------------------------------
 def time_launches(torch, fn, n_iter, n_warm=3):
-    """Average device milliseconds of fn(i) over n_iter launches (CUDA events on the current stream)."""
+    """Average device milliseconds of fn(i) over n_iter launches (CUDA events on the launching stream).
+
+    The launches are captured once into a CUDA graph and the graph is replayed for the timed run, so that
+    launches far shorter than the host's launch cost (a 1 MiB softmax) are limited by the device, not by
+    Python; if capture is not possible the launches are issued directly."""
     for i in range(n_warm):
         fn(i)
     torch.cuda.synchronize()
+    graph = None
+    try:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(n_iter):
+                    fn(n_warm + i)
+        torch.cuda.current_stream().wait_stream(side)
+        graph = g
+    except Exception:
+        graph = None
+        torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(n_iter):
-        fn(n_warm + i)
-    e1.record()
+    if graph is not None:
+        graph.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        graph.replay()
+        e1.record()
+    else:
+        e0.record()
+        for i in range(n_iter):
+            fn(n_warm + i)
+        e1.record()
     torch.cuda.synchronize()
     return e0.elapsed_time(e1) / n_iter
 
@@ -248,6 +273,11 @@ def ops_suite(torch, api, peaks, only: str = ""):
                                           "frac_measured_sustained": tf / peaks["bf16_tflops_sustained"],
                                           "frac_nominal": tf / NOMINAL_BF16_TFLOPS, "note": "configured shape"}
         del cs
+    # the vendor library on the same shape, same timing method: context only, never on the product path
+    cs = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    ms = time_launches(torch, lambda i: torch.matmul(as_[i % 3], bs[i % 3], out=cs[i % 3]), 30)
+    out[f"context_cublas_{M}x{N}x{K}_cbf16"] = {"ms": ms, "TFLOP/s": 2.0 * M * N * K / ms / 1e9,
+                                               "note": "torch.matmul (cuBLAS), for context: not part of the library"}
     return out
 
 

@@ -8,7 +8,7 @@
 // registers (data centred before squaring, mean refined by the mean of the
 // residuals: no E[x^2] - mu^2 cancellation), reduced with warp shuffles.
 //   * cols <= 1024   : one warp per row
-//   * cols <= 16384  : one CTA of 512 threads per row
+//   * cols <= 16384  : one CTA of 64 to 512 threads per row
 //   * otherwise      : one CTA per row, three passes from global/L2; partial
 //                      statistics are merged pairwise (Chan/Welford form)
 #include "pd_common.cuh"
@@ -131,17 +131,21 @@ template <int VPT, typename OutT>
 void launch_warp_rows(const float* x, const float* g, const float* b, OutT* y, int64_t rows, int cols, float eps,
                       cudaStream_t s) {
   constexpr int kThreads = 256, kRowsPerCta = kThreads / 32;
+  auto kernel = layernorm_rows_in_registers<VPT, 32, kThreads, OutT>;
+  // one CTA per eight rows, all launched: the hardware scheduler balances many short CTAs better than a
+  // grid-stride loop over a resident set does
   const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
-  const int grid = (int)(ctas < (int64_t)sm_count() * 64 ? ctas : (int64_t)sm_count() * 64);
-  layernorm_rows_in_registers<VPT, 32, kThreads, OutT><<<grid, kThreads, 0, s>>>(x, g, b, y, rows, cols, eps);
+  const int grid = (int)(ctas < 0x7fffffff ? ctas : 0x7fffffff);
+  kernel<<<grid, kThreads, 0, s>>>(x, g, b, y, rows, cols, eps);
 }
 
-template <int VPT, typename OutT>
+// One CTA of THREADS threads per row, up to 8 float4 per thread.
+template <int THREADS, typename OutT>
 void launch_cta_rows(const float* x, const float* g, const float* b, OutT* y, int64_t rows, int cols, float eps,
                      cudaStream_t s) {
-  constexpr int kThreads = 512;
-  const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
-  layernorm_rows_in_registers<VPT, kThreads, kThreads, OutT><<<grid, kThreads, 0, s>>>(x, g, b, y, rows, cols, eps);
+  auto kernel = layernorm_rows_in_registers<8, THREADS, THREADS, OutT>;
+  const int grid = (int)(rows < 0x7fffffff ? rows : 0x7fffffff);
+  kernel<<<grid, THREADS, 0, s>>>(x, g, b, y, rows, cols, eps);
 }
 
 template <typename OutT>
@@ -157,10 +161,10 @@ pd_status dispatch(const float* x, const float* g, const float* b, OutT* y, int6
     else launch_warp_rows<8>(x, g, b, y, rows, c, eps, s);
   } else if (vec_ok && cols <= 16384) {
     const int c = (int)cols;
-    if (c <= 2048) launch_cta_rows<1>(x, g, b, y, rows, c, eps, s);
-    else if (c <= 4096) launch_cta_rows<2>(x, g, b, y, rows, c, eps, s);
-    else if (c <= 8192) launch_cta_rows<4>(x, g, b, y, rows, c, eps, s);
-    else launch_cta_rows<8>(x, g, b, y, rows, c, eps, s);
+    if (c <= 2048) launch_cta_rows<64>(x, g, b, y, rows, c, eps, s);
+    else if (c <= 4096) launch_cta_rows<128>(x, g, b, y, rows, c, eps, s);
+    else if (c <= 8192) launch_cta_rows<256>(x, g, b, y, rows, c, eps, s);
+    else launch_cta_rows<512>(x, g, b, y, rows, c, eps, s);
   } else {
     const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
     layernorm_rows_generic<OutT><<<grid, 256, 0, s>>>(x, g, b, y, rows, cols, eps);

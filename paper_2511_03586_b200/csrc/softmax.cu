@@ -6,7 +6,7 @@
 // global memory exactly once into registers with 128-bit loads, reduced with
 // warp shuffles, and written once.
 //   * cols <= 1024            : one warp per row (up to 8 float4 per lane)
-//   * cols <= 16384           : one CTA of 512 threads per row (up to 8 float4 per thread)
+//   * cols <= 16384           : one CTA of 64 to 512 threads per row (8 float4 per thread)
 //   * anything else / ragged  : one CTA per row, three passes from global/L2
 #include "pd_common.cuh"
 
@@ -83,16 +83,20 @@ softmax_rows_generic(const float* __restrict__ x, OutT* __restrict__ y, int64_t 
 template <int VPT, typename OutT>
 void launch_warp_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStream_t s) {
   constexpr int kThreads = 256, kRowsPerCta = kThreads / 32;
+  auto kernel = softmax_rows_in_registers<VPT, 32, kThreads, OutT>;
+  // one CTA per eight rows, all launched: the hardware scheduler balances many short CTAs better than a
+  // grid-stride loop over a resident set does
   const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
-  const int grid = (int)(ctas < (int64_t)sm_count() * 64 ? ctas : (int64_t)sm_count() * 64);
-  softmax_rows_in_registers<VPT, 32, kThreads, OutT><<<grid, kThreads, 0, s>>>(x, y, rows, cols);
+  const int grid = (int)(ctas < 0x7fffffff ? ctas : 0x7fffffff);
+  kernel<<<grid, kThreads, 0, s>>>(x, y, rows, cols);
 }
 
-template <int VPT, typename OutT>
+// One CTA of THREADS threads per row, up to 8 float4 per thread.
+template <int THREADS, typename OutT>
 void launch_cta_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStream_t s) {
-  constexpr int kThreads = 512;
-  const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
-  softmax_rows_in_registers<VPT, kThreads, kThreads, OutT><<<grid, kThreads, 0, s>>>(x, y, rows, cols);
+  auto kernel = softmax_rows_in_registers<8, THREADS, THREADS, OutT>;
+  const int grid = (int)(rows < 0x7fffffff ? rows : 0x7fffffff);
+  kernel<<<grid, THREADS, 0, s>>>(x, y, rows, cols);
 }
 
 template <typename OutT>
@@ -106,10 +110,10 @@ pd_status dispatch(const float* x, OutT* y, int64_t rows, int64_t cols, cudaStre
     else launch_warp_rows<8>(x, y, rows, c, s);
   } else if (vec_ok && cols <= 16384) {
     const int c = (int)cols;
-    if (c <= 2048) launch_cta_rows<1>(x, y, rows, c, s);
-    else if (c <= 4096) launch_cta_rows<2>(x, y, rows, c, s);
-    else if (c <= 8192) launch_cta_rows<4>(x, y, rows, c, s);
-    else launch_cta_rows<8>(x, y, rows, c, s);
+    if (c <= 2048) launch_cta_rows<64>(x, y, rows, c, s);
+    else if (c <= 4096) launch_cta_rows<128>(x, y, rows, c, s);
+    else if (c <= 8192) launch_cta_rows<256>(x, y, rows, c, s);
+    else launch_cta_rows<512>(x, y, rows, c, s);
   } else {
     const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
     softmax_rows_generic<OutT><<<grid, 256, 0, s>>>(x, y, rows, cols);
