@@ -148,6 +148,9 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   __syncthreads();
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above is independent of other kernels' data; from here on global memory is touched
+  griddep_wait();
+  griddep_launch_dependents();
 
   // Work decomposition shared by all roles: unit -> (batch, head, first query block, active slots).
   auto unit_coords = [&](int unit, int& b, int& h, int& qb0, int& nslots) {
@@ -488,7 +491,7 @@ pd_status launch_fused_attention(const __nv_bfloat16* qkv, __nv_bfloat16* ctx, i
     attr_set = true;
   }
   const int grid = p.num_units < sm_count() ? p.num_units : sm_count();
-  attention_fwd_tcgen05_kernel<<<grid, kThreads, kSmemBytes, s>>>(tq, tk, tv, to, p);
+  launch_pdl(attention_fwd_tcgen05_kernel, dim3(grid), dim3(kThreads), kSmemBytes, s, tq, tk, tv, to, p);
   return check_launch();
 }
 

@@ -91,6 +91,9 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   __syncthreads();
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above is independent of other kernels' data; from here on global memory is touched
+  griddep_wait();
+  griddep_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
@@ -222,7 +225,7 @@ pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
     attr_set = true;
   }
   const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
-  kernel<<<grid, kThreads, C::kSmemBytes, s>>>(ta, tb, tc, p);
+  launch_pdl(kernel, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, tc, p);
   return check_launch();
 }
 

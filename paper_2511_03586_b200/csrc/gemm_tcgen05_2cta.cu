@@ -86,6 +86,9 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
   cluster_sync_all();  // barriers of both CTAs are initialised before anyone signals them
   tcgen05_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // everything above is independent of other kernels' data; from here on global memory is touched
+  griddep_wait();
+  griddep_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
@@ -219,7 +222,7 @@ pd_status launch_pair_variant(const GemmProblem& g, cudaStream_t s) {
     attr_set = true;
   }
   const int pairs = (int)(tiles < sm_count() / 2 ? tiles : sm_count() / 2);
-  kernel<<<2 * pairs, kThreads, kSmemBytes, s>>>(ta, tb, tc, p);
+  launch_pdl(kernel, dim3(2 * pairs), dim3(kThreads), kSmemBytes, s, ta, tb, tc, p);
   return check_launch();
 }
 

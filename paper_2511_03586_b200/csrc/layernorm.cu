@@ -29,6 +29,8 @@ layernorm_rows_in_registers(const float* __restrict__ x, const float* __restrict
   const float inv_cols = 1.0f / (float)cols;
   const float4* g4 = reinterpret_cast<const float4*>(gamma);
   const float4* b4 = reinterpret_cast<const float4*>(beta);
+  griddep_wait();
+  griddep_launch_dependents();
   for (int64_t row = (int64_t)blockIdx.x * ROWS_PER_CTA + threadIdx.x / THREADS_PER_ROW; row < rows;
        row += (int64_t)gridDim.x * ROWS_PER_CTA) {
     const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
@@ -136,7 +138,7 @@ void launch_warp_rows(const float* x, const float* g, const float* b, OutT* y, i
   // grid-stride loop over a resident set does
   const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
   const int grid = (int)(ctas < 0x7fffffff ? ctas : 0x7fffffff);
-  kernel<<<grid, kThreads, 0, s>>>(x, g, b, y, rows, cols, eps);
+  launch_pdl(kernel, dim3(grid), dim3(kThreads), 0, s, x, g, b, y, rows, cols, eps);
 }
 
 // One CTA of THREADS threads per row, up to 8 float4 per thread.
@@ -145,7 +147,7 @@ void launch_cta_rows(const float* x, const float* g, const float* b, OutT* y, in
                      cudaStream_t s) {
   auto kernel = layernorm_rows_in_registers<8, THREADS, THREADS, OutT>;
   const int grid = (int)(rows < 0x7fffffff ? rows : 0x7fffffff);
-  kernel<<<grid, THREADS, 0, s>>>(x, g, b, y, rows, cols, eps);
+  launch_pdl(kernel, dim3(grid), dim3(THREADS), 0, s, x, g, b, y, rows, cols, eps);
 }
 
 template <typename OutT>

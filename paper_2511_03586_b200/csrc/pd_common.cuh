@@ -23,9 +23,35 @@ int sm_count();
 // Device address of the status word the bounded waits report to (nullptr on failure).
 int* device_status_ptr();
 
+// Launch with programmatic stream serialisation: the kernel may become resident and run its prologue while the
+// previous kernel of the stream is still draining; it must call griddep_wait() before it touches global memory
+// that an earlier kernel may still read or write.  Kernels call griddep_launch_dependents() to let their own
+// successor do the same.
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                       Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ---- device side ---------------------------------------------------------
+// Blocks until every kernel this one depends on has completed and its writes are visible (no-op when the
+// kernel was launched without programmatic serialisation).
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Allows the next kernel of the stream to be scheduled as soon as resources free up.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));

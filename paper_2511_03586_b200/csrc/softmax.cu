@@ -26,6 +26,8 @@ softmax_rows_in_registers(const float* __restrict__ x, OutT* __restrict__ y, int
   __shared__ float scratch[2][NWARPS];
   const int t = threadIdx.x % THREADS_PER_ROW;
   const int cols4 = cols >> 2;
+  griddep_wait();
+  griddep_launch_dependents();
   for (int64_t row = (int64_t)blockIdx.x * ROWS_PER_CTA + threadIdx.x / THREADS_PER_ROW; row < rows;
        row += (int64_t)gridDim.x * ROWS_PER_CTA) {
     const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
@@ -88,7 +90,7 @@ void launch_warp_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStrea
   // grid-stride loop over a resident set does
   const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
   const int grid = (int)(ctas < 0x7fffffff ? ctas : 0x7fffffff);
-  kernel<<<grid, kThreads, 0, s>>>(x, y, rows, cols);
+  launch_pdl(kernel, dim3(grid), dim3(kThreads), 0, s, x, y, rows, cols);
 }
 
 // One CTA of THREADS threads per row, up to 8 float4 per thread.
@@ -96,7 +98,7 @@ template <int THREADS, typename OutT>
 void launch_cta_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStream_t s) {
   auto kernel = softmax_rows_in_registers<8, THREADS, THREADS, OutT>;
   const int grid = (int)(rows < 0x7fffffff ? rows : 0x7fffffff);
-  kernel<<<grid, THREADS, 0, s>>>(x, y, rows, cols);
+  launch_pdl(kernel, dim3(grid), dim3(THREADS), 0, s, x, y, rows, cols);
 }
 
 template <typename OutT>
