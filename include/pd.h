@@ -79,6 +79,13 @@ pd_status pd_softmax(const float* x, float* y, int64_t rows, int64_t cols, cudaS
 pd_status pd_layernorm(const float* x, const float* gamma, const float* beta, float* y,
                        int64_t rows, int64_t cols, float eps, cudaStream_t stream);
 
+/* Root-mean-square normalisation over the last dimension (operator "rmsnorm" of
+ * the paper's table, 3072 x 4096):
+ *   y[i,j] = x[i,j] / sqrt(mean_j x[i,j]^2 + eps) * gamma[j].
+ * x, y: fp32 [rows, cols]; gamma: fp32 [cols].  y may alias x. */
+pd_status pd_rmsnorm(const float* x, const float* gamma, float* y, int64_t rows, int64_t cols, float eps,
+                     cudaStream_t stream);
+
 /* Fused bias + GELU(erf) + residual in one pass over HBM (element-wise and
  * broadcast features; nearest paper operators "add" and "relu"):
  *   out[i,j] = GELU(x[i,j] + bias[j]) + r[i,j],  GELU(z) = z/2 * (1 + erf(z/sqrt 2)).

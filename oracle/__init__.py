@@ -38,6 +38,8 @@ def _load():
         lib = ctypes.CDLL(build())
         lib.oracle_softmax.argtypes = [_D, _D, _I64, _I64]
         lib.oracle_layernorm.argtypes = [_D, _D, _D, _D, _I64, _I64, ctypes.c_double]
+        lib.oracle_rmsnorm.argtypes = [_D, _D, _D, _I64, _I64, ctypes.c_double]
+        lib.oracle_rmsnorm.restype = ctypes.c_int
         lib.oracle_bias_gelu_residual.argtypes = [_D, _D, _D, _D, _I64, _I64]
         lib.oracle_gemm.argtypes = [_D, _D, _D, _I64, _I64, _I64]
         lib.oracle_attention.argtypes = [_D, _D, _D, _I64, _I64, _I64, _I64]
@@ -76,6 +78,15 @@ def layernorm(x, gamma, beta, eps: float) -> np.ndarray:
     assert gamma.shape == (cols,) and beta.shape == (cols,)
     y = np.empty_like(x)
     _check(_load().oracle_layernorm(_p(x), _p(gamma), _p(beta), _p(y), rows, cols, float(eps)), "oracle_layernorm")
+    return y
+
+
+def rmsnorm(x, gamma, eps: float) -> np.ndarray:
+    x, gamma = _f64(x), _f64(gamma)
+    rows, cols = x.shape
+    assert gamma.shape == (cols,)
+    y = np.empty_like(x)
+    _check(_load().oracle_rmsnorm(_p(x), _p(gamma), _p(y), rows, cols, float(eps)), "oracle_rmsnorm")
     return y
 
 

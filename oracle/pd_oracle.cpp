@@ -23,6 +23,7 @@
 //   layernorm  N M  mu[i] += x[i,j] / M
 //              N M  v[i]  += (x[i,j] - mu[i])^2 / M          (biased variance)
 //              N M  y[i,j] = (x[i,j] - mu[i]) / sqrt(v[i] + eps) * g[j] + b[j]
+//   rmsnorm    N M  q[i]  += x[i,j]^2 / M;  y[i,j] = x[i,j] / sqrt(q[i] + eps) * g[j]
 //   bias_gelu  N M  z = x[i,j] + bias[j]
 //                   out[i,j] = 0.5 * z * (1 + erf(z / sqrt(2))) + r[i,j]
 //   gemm       M N K  c[m,n] += a[m,k] * b[k,n]
@@ -75,6 +76,22 @@ int oracle_layernorm(const double* x, const double* gamma, const double* beta, d
     for (int64_t j = 0; j < cols; ++j) v += (xi[j] - mu) * (xi[j] - mu) / M;
     const double denom = std::sqrt(v + eps);
     for (int64_t j = 0; j < cols; ++j) yi[j] = (xi[j] - mu) / denom * gamma[j] + beta[j];
+  }
+  return 0;
+}
+
+// Root-mean-square normalisation over the last dimension (operator "rmsnorm"):
+//   N M  q[i]  += x[i,j]^2 / M
+//   N M  y[i,j] = x[i,j] / sqrt(q[i] + eps) * g[j]
+int oracle_rmsnorm(const double* x, const double* gamma, double* y, int64_t rows, int64_t cols, double eps) {
+  if (!x || !gamma || !y || rows < 0 || cols <= 0) return -1;
+  const double M = static_cast<double>(cols);
+  for (int64_t i = 0; i < rows; ++i) {
+    const double* xi = x + i * cols;
+    double q = 0.0;
+    for (int64_t j = 0; j < cols; ++j) q += xi[j] * xi[j] / M;
+    const double denom = std::sqrt(q + eps);
+    for (int64_t j = 0; j < cols; ++j) y[i * cols + j] = xi[j] / denom * gamma[j];
   }
   return 0;
 }

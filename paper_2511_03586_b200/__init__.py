@@ -7,7 +7,7 @@ imports without the CUDA library; everything else lives in
 """
 import importlib
 
-__all__ = ["api", "inputs", "build"]
+__all__ = ["api", "inputs", "build", "replicas"]
 
 
 def __getattr__(name):

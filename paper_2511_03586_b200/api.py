@@ -22,7 +22,7 @@ PD_BF16, PD_F32 = 0, 1
 
 EXPORTS = (
     "pd_status_string", "pd_last_cuda_error", "pd_get_device_status", "pd_clear_device_status",
-    "pd_softmax", "pd_layernorm", "pd_bias_gelu_residual", "pd_gemm_bf16", "pd_set_gemm_tile_mode", "pd_attention_fwd",
+    "pd_softmax", "pd_layernorm", "pd_rmsnorm", "pd_bias_gelu_residual", "pd_gemm_bf16", "pd_set_gemm_tile_mode", "pd_attention_fwd",
     "pd_encoder_layer_workspace_bytes", "pd_encoder_layer_fwd", "pd_encoder_layer_stage_count",
     "pd_encoder_layer_stage_name", "pd_encoder_layer_fwd_profiled", "pd_encoder_layer_static_scratch_bytes",
     "pd_encoder_layer_fwd_static",
@@ -59,6 +59,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_clear_device_status.argtypes = []; lib.pd_clear_device_status.restype = st
     lib.pd_softmax.argtypes = [vp, vp, i64, i64, vp]; lib.pd_softmax.restype = st
     lib.pd_layernorm.argtypes = [vp, vp, vp, vp, i64, i64, ctypes.c_float, vp]; lib.pd_layernorm.restype = st
+    lib.pd_rmsnorm.argtypes = [vp, vp, vp, i64, i64, ctypes.c_float, vp]; lib.pd_rmsnorm.restype = st
     lib.pd_bias_gelu_residual.argtypes = [vp, vp, vp, vp, i64, i64, vp]; lib.pd_bias_gelu_residual.restype = st
     lib.pd_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, ctypes.c_int, ctypes.c_int,
                                  i64, i64, i64, i64, vp]
@@ -121,6 +122,15 @@ def pd_layernorm(x, gamma, beta, eps: float, y=None, stream=None) -> torch.Tenso
     _check(_lib.pd_layernorm(_dev(x, torch.float32, "x"), _dev(gamma, torch.float32, "gamma"),
                              _dev(beta, torch.float32, "beta"), _dev(y, torch.float32, "y"), rows, cols,
                              float(eps), _stream(stream)), "pd_layernorm")
+    return y
+
+
+def pd_rmsnorm(x, gamma, eps: float, y=None, stream=None) -> torch.Tensor:
+    rows, cols = x.shape
+    if y is None:
+        y = torch.empty_like(x)
+    _check(_lib.pd_rmsnorm(_dev(x, torch.float32, "x"), _dev(gamma, torch.float32, "gamma"),
+                           _dev(y, torch.float32, "y"), rows, cols, float(eps), _stream(stream)), "pd_rmsnorm")
     return y
 
 

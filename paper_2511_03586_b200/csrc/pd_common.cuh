@@ -105,6 +105,8 @@ pd_status launch_softmax(const float* x, void* y, bool y_is_bf16, int64_t rows, 
 // LayerNorm with fp32 or bf16 output.
 pd_status launch_layernorm(const float* x, const float* gamma, const float* beta, void* y, bool y_is_bf16,
                            int64_t rows, int64_t cols, float eps, cudaStream_t s);
+pd_status launch_rmsnorm(const float* x, const float* gamma, float* y, int64_t rows, int64_t cols, float eps,
+                         cudaStream_t s);
 pd_status launch_bias_gelu_residual(const float* x, const float* bias, const float* r, float* out,
                                     int64_t rows, int64_t cols, cudaStream_t s);
 

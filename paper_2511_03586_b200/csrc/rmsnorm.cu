@@ -1,0 +1,117 @@
+// Root-mean-square normalisation over the last dimension, fp32 in, fp32 out
+// (operator "rmsnorm" of the paper's operator table, 3072 x 4096):
+//
+//   y[i,j] = x[i,j] * rsqrt(mean_j x[i,j]^2 + eps) * gamma[j]
+//
+// HBM-bound, 8 bytes per element: the row is read once into registers with
+// 128-bit streaming loads, the sum of squares is reduced with warp shuffles (and
+// through shared memory when several warps share a row), and the row is written
+// once.  Same three paths as the LayerNorm kernel.
+#include "pd_common.cuh"
+
+namespace pd {
+namespace {
+
+template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA>
+__global__ void __launch_bounds__(THREADS_PER_CTA)
+rmsnorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__ gamma, float* __restrict__ y,
+                          int64_t rows, int cols, float eps) {
+  constexpr int ROWS_PER_CTA = THREADS_PER_CTA / THREADS_PER_ROW;
+  constexpr int NWARPS = THREADS_PER_ROW / 32;
+  __shared__ float scratch[2][NWARPS];
+  const int t = threadIdx.x % THREADS_PER_ROW;
+  const int cols4 = cols >> 2;
+  const float inv_cols = 1.0f / (float)cols;
+  const float4* g4 = reinterpret_cast<const float4*>(gamma);
+  griddep_wait();
+  griddep_launch_dependents();
+  int slot = 0;
+  for (int64_t row = (int64_t)blockIdx.x * ROWS_PER_CTA + threadIdx.x / THREADS_PER_ROW; row < rows;
+       row += (int64_t)gridDim.x * ROWS_PER_CTA, slot ^= 1) {
+    const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
+    float4 v[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int c = t + i * THREADS_PER_ROW;
+      v[i] = (c < cols4) ? ld_stream(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) q += (v[i].x * v[i].x + v[i].y * v[i].y) + (v[i].z * v[i].z + v[i].w * v[i].w);
+    const float rstd = rsqrtf(block_reduce<NWARPS, false>(q, scratch, slot) * inv_cols + eps);
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int c = t + i * THREADS_PER_ROW;
+      if (c < cols4) {
+        const float4 g = __ldg(g4 + c);
+        store_out4(y, row * cols4 + c,
+                   make_float4(v[i].x * rstd * g.x, v[i].y * rstd * g.y, v[i].z * rstd * g.z, v[i].w * rstd * g.w));
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256)
+rmsnorm_rows_generic(const float* __restrict__ x, const float* __restrict__ gamma, float* __restrict__ y,
+                     int64_t rows, int64_t cols, float eps) {
+  __shared__ float scratch[2][8];
+  int slot = 0;
+  for (int64_t row = blockIdx.x; row < rows; row += gridDim.x, slot ^= 1) {
+    const float* xr = x + row * cols;
+    float q = 0.f;
+    for (int64_t j = threadIdx.x; j < cols; j += 256) q += xr[j] * xr[j];
+    const float rstd = rsqrtf(block_reduce<8, false>(q, scratch, slot) / (float)cols + eps);
+    for (int64_t j = threadIdx.x; j < cols; j += 256) y[row * cols + j] = xr[j] * rstd * gamma[j];
+  }
+}
+
+template <int VPT>
+void launch_warp_rows(const float* x, const float* g, float* y, int64_t rows, int cols, float eps, cudaStream_t s) {
+  constexpr int kThreads = 256, kRowsPerCta = kThreads / 32;
+  const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
+  const int grid = (int)(ctas < 0x7fffffff ? ctas : 0x7fffffff);
+  launch_pdl(rmsnorm_rows_in_registers<VPT, 32, kThreads>, dim3(grid), dim3(kThreads), 0, s, x, g, y, rows, cols, eps);
+}
+
+template <int THREADS>
+void launch_cta_rows(const float* x, const float* g, float* y, int64_t rows, int cols, float eps, cudaStream_t s) {
+  const int grid = (int)(rows < 0x7fffffff ? rows : 0x7fffffff);
+  launch_pdl(rmsnorm_rows_in_registers<8, THREADS, THREADS>, dim3(grid), dim3(THREADS), 0, s, x, g, y, rows, cols, eps);
+}
+
+}  // namespace
+
+pd_status launch_rmsnorm(const float* x, const float* g, float* y, int64_t rows, int64_t cols, float eps,
+                         cudaStream_t s) {
+  const bool vec_ok = (cols % 4 == 0) && aligned16(x) && aligned16(g) && aligned16(y);
+  const int c = (int)cols;
+  if (vec_ok && cols <= 1024) {
+    if (c <= 128) launch_warp_rows<1>(x, g, y, rows, c, eps, s);
+    else if (c <= 256) launch_warp_rows<2>(x, g, y, rows, c, eps, s);
+    else if (c <= 512) launch_warp_rows<4>(x, g, y, rows, c, eps, s);
+    else launch_warp_rows<8>(x, g, y, rows, c, eps, s);
+  } else if (vec_ok && cols <= 16384) {
+    if (c <= 2048) launch_cta_rows<64>(x, g, y, rows, c, eps, s);
+    else if (c <= 4096) launch_cta_rows<128>(x, g, y, rows, c, eps, s);
+    else if (c <= 8192) launch_cta_rows<256>(x, g, y, rows, c, eps, s);
+    else launch_cta_rows<512>(x, g, y, rows, c, eps, s);
+  } else {
+    const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
+    rmsnorm_rows_generic<<<grid, 256, 0, s>>>(x, g, y, rows, cols, eps);
+  }
+  return check_launch();
+}
+
+}  // namespace pd
+
+extern "C" pd_status pd_rmsnorm(const float* x, const float* gamma, float* y, int64_t rows, int64_t cols, float eps,
+                                cudaStream_t stream) {
+  if (!x || !gamma || !y) return PD_ERR_NULL_POINTER;
+  if (rows < 0 || cols <= 0 || !(eps >= 0.f)) return PD_ERR_BAD_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(y) | reinterpret_cast<uintptr_t>(gamma)) & 3u)
+    return PD_ERR_ALIGNMENT;
+  if (rows == 0) return PD_OK;
+  pd_status st = pd::require_sm100();
+  if (st != PD_OK) return st;
+  return pd::launch_rmsnorm(x, gamma, y, rows, cols, eps, stream);
+}

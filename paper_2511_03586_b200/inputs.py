@@ -75,6 +75,12 @@ def layernorm_inputs(rows: int, cols: int, seed: int = 0):
     return {"x": x, "gamma": gamma, "beta": beta, "eps": 1e-5}
 
 
+def rmsnorm_inputs(rows: int, cols: int, seed: int = 0):
+    """X ~ N(1, 2); gamma ~ U(0.5, 1.5); fp32 (the layernorm recipe without beta)."""
+    rng = _rng(seed)
+    return {"x": _normal(rng, (rows, cols), 1.0, 2.0), "gamma": _uniform(rng, (cols,), 0.5, 1.5), "eps": 1e-5}
+
+
 def bias_gelu_residual_inputs(rows: int, cols: int, seed: int = 0):
     """X, R ~ N(0, 1) fp32 [rows, cols]; bias ~ N(0, 0.02) fp32 [cols]."""
     rng = _rng(seed)

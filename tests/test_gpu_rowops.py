@@ -98,6 +98,27 @@ def test_layernorm_large_mean_is_stable(api):
 
 
 @pytest.mark.parametrize("cols", COLS)
+def test_rmsnorm_shapes(api, cols):
+    for rows in ROWS:
+        p = inputs.rmsnorm_inputs(rows, cols, seed=rows)
+        y = Guarded((rows, cols), torch.float32)
+        api.pd_rmsnorm(dev_f32(p["x"]), dev_f32(p["gamma"]), p["eps"], y.t)
+        torch.cuda.synchronize()
+        y.check()
+        assert max_rel(host(y.t), oracle.rmsnorm(p["x"], p["gamma"], np.float32(p["eps"]))) < TOL
+
+
+def test_rmsnorm_paper_shape_and_in_place(api):
+    rows, cols = 3072, 4096                       # Table "ML operators optimized using PerfLLM": rmsnorm
+    p = inputs.rmsnorm_inputs(rows, cols, seed=0)
+    xd, gd = dev_f32(p["x"]), dev_f32(p["gamma"])
+    y = api.pd_rmsnorm(xd, gd, p["eps"])
+    assert max_rel(host(y), oracle.rmsnorm(p["x"], p["gamma"], np.float32(p["eps"]))) < TOL
+    api.pd_rmsnorm(xd, gd, p["eps"], xd)
+    assert torch.equal(xd, y)
+
+
+@pytest.mark.parametrize("cols", COLS)
 def test_bias_gelu_residual_shapes(api, cols):
     for rows in ROWS:
         p = inputs.bias_gelu_residual_inputs(rows, cols, seed=rows)

@@ -127,6 +127,32 @@ def test_layernorm_constant_row_gives_beta():
     assert np.array_equal(y, np.tile(b, (2, 1)))
 
 
+# ------------------------------------------------------------------ rmsnorm
+def test_rmsnorm_closed_forms_and_invariants():
+    # constant row c: y = c / sqrt(c^2 + eps) * gamma
+    g = np.linspace(0.5, 1.5, 8)
+    y = oracle.rmsnorm(np.full((2, 8), -3.0), g, 7.0)
+    np.testing.assert_allclose(y, np.tile(-3.0 / 4.0 * g, (2, 1)), rtol=1e-15)
+    # row (3, 4): mean square 12.5 -> y = x / sqrt(12.5)
+    np.testing.assert_allclose(oracle.rmsnorm(np.array([[3.0, 4.0]]), np.ones(2), 0.0),
+                               [[3 / math.sqrt(12.5), 4 / math.sqrt(12.5)]], rtol=1e-15)
+    rng = np.random.default_rng(40)
+    x = rng.normal(1, 2, size=(5, 33))
+    y = oracle.rmsnorm(x, np.ones(33), 0.0)
+    np.testing.assert_allclose((y * y).mean(axis=1), 1.0, rtol=1e-13)          # unit mean square
+    np.testing.assert_allclose(oracle.rmsnorm(4.0 * x, np.ones(33), 0.0), y, rtol=1e-12)   # scale invariant
+    assert not np.allclose(oracle.rmsnorm(x + 1.0, np.ones(33), 0.0), y)       # but not shift invariant
+    # on a zero-mean row it coincides with layernorm (beta = 0)
+    xc = x - x.mean(axis=1, keepdims=True)
+    g = rng.uniform(0.5, 1.5, 33)
+    np.testing.assert_allclose(oracle.rmsnorm(xc, g, 1e-5), oracle.layernorm(xc, g, np.zeros(33), 1e-5),
+                               rtol=1e-10, atol=1e-12)
+    # gamma is indexed by column
+    g2 = g.copy(); g2[4] = 9.0
+    changed = np.where(np.any(oracle.rmsnorm(x, g2, 1e-5) != oracle.rmsnorm(x, g, 1e-5), axis=0))[0]
+    assert list(changed) == [4]
+
+
 # ------------------------------------------------------- bias + GELU + residual
 def _erf_series(x: float) -> float:
     """erf by its Maclaurin series 2/sqrt(pi) * sum (-1)^n x^(2n+1) / (n! (2n+1)),
