@@ -8,8 +8,10 @@
 // registers (data centred before squaring, mean refined by the mean of the
 // residuals: no E[x^2] - mu^2 cancellation), reduced with warp shuffles.
 //   * cols <= 1024   : one warp per row
-//   * cols <= 16384  : one CTA of 64 to 512 threads per row
-//   * otherwise      : one CTA per row, three passes from global/L2; partial
+//   * cols <= 32768  : one CTA of 64 to 1024 threads per row
+//   * longer, aligned: one CTA per row, three 128-bit passes (mean from HBM; centred
+//                      second moment and normalisation from L2)
+//   * otherwise      : one CTA per row, three scalar passes from global/L2; partial
 //                      statistics are merged pairwise (Chan/Welford form)
 #include "pd_common.cuh"
 
@@ -17,7 +19,7 @@ namespace pd {
 namespace {
 
 template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA, typename OutT>
-__global__ void __launch_bounds__(THREADS_PER_CTA)
+__global__ void __launch_bounds__(THREADS_PER_CTA, THREADS_PER_CTA >= 1024 ? 1 : 1024 / THREADS_PER_CTA)  // at most 64 registers: 1024 threads resident per SM
 layernorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__ gamma,
                             const float* __restrict__ beta, OutT* __restrict__ y, int64_t rows, int cols,
                             float eps) {
@@ -129,6 +131,47 @@ layernorm_rows_generic(const float* __restrict__ x, const float* __restrict__ ga
   }
 }
 
+// Rows too long for registers (cols > 32768), 16-byte aligned: one CTA of 512 threads per row, three passes with
+// 128-bit accesses: mean (from HBM), centred second moment and normalisation (both from L2, where the row still is).
+template <typename OutT>
+__global__ void __launch_bounds__(512)
+layernorm_rows_streaming(const float* __restrict__ x, const float* __restrict__ gamma,
+                         const float* __restrict__ beta, OutT* __restrict__ y, int64_t rows, int64_t cols,
+                         float eps) {
+  __shared__ float scratch[3][16];
+  const int64_t cols4 = cols >> 2;
+  const float inv_cols = 1.0f / (float)cols;
+  const float4* g4 = reinterpret_cast<const float4*>(gamma);
+  const float4* b4 = reinterpret_cast<const float4*>(beta);
+  for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+    const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
+    const float shift = __ldg(reinterpret_cast<const float*>(xr));  // keeps the first sum small when |mean| >> spread
+    float s = 0.f;
+    for (int64_t c = threadIdx.x; c < cols4; c += 512) {
+      const float4 v = __ldg(xr + c);
+      s += ((v.x - shift) + (v.y - shift)) + ((v.z - shift) + (v.w - shift));
+    }
+    const float mu = shift + block_reduce<16, false>(s, scratch, 0) * inv_cols;
+    float q = 0.f, d1 = 0.f;
+    for (int64_t c = threadIdx.x; c < cols4; c += 512) {
+      const float4 v = __ldg(xr + c);
+      const float a = v.x - mu, b = v.y - mu, cc = v.z - mu, d = v.w - mu;
+      d1 += (a + b) + (cc + d);
+      q += (a * a + b * b) + (cc * cc + d * d);
+    }
+    const float delta = block_reduce<16, false>(d1, scratch, 1) * inv_cols;  // residual of the mean
+    const float var = fmaxf(block_reduce<16, false>(q, scratch, 2) * inv_cols - delta * delta, 0.f);
+    const float rstd = rsqrtf(var + eps);  // (v - mu) - delta below: adding delta to mu would round it away
+    for (int64_t c = threadIdx.x; c < cols4; c += 512) {
+      const float4 v = __ldg(xr + c), g = __ldg(g4 + c), b = __ldg(b4 + c);
+      store_out4(y, row * cols4 + c,
+                 make_float4(((v.x - mu) - delta) * rstd * g.x + b.x, ((v.y - mu) - delta) * rstd * g.y + b.y,
+                             ((v.z - mu) - delta) * rstd * g.z + b.z, ((v.w - mu) - delta) * rstd * g.w + b.w));
+    }
+    __syncthreads();
+  }
+}
+
 template <int VPT, typename OutT>
 void launch_warp_rows(const float* x, const float* g, const float* b, OutT* y, int64_t rows, int cols, float eps,
                       cudaStream_t s) {
@@ -161,12 +204,16 @@ pd_status dispatch(const float* x, const float* g, const float* b, OutT* y, int6
     else if (c <= 256) launch_warp_rows<2>(x, g, b, y, rows, c, eps, s);
     else if (c <= 512) launch_warp_rows<4>(x, g, b, y, rows, c, eps, s);
     else launch_warp_rows<8>(x, g, b, y, rows, c, eps, s);
-  } else if (vec_ok && cols <= 16384) {
+  } else if (vec_ok && cols <= 32768) {
     const int c = (int)cols;
     if (c <= 2048) launch_cta_rows<64>(x, g, b, y, rows, c, eps, s);
     else if (c <= 4096) launch_cta_rows<128>(x, g, b, y, rows, c, eps, s);
     else if (c <= 8192) launch_cta_rows<256>(x, g, b, y, rows, c, eps, s);
-    else launch_cta_rows<512>(x, g, b, y, rows, c, eps, s);
+    else if (c <= 16384) launch_cta_rows<512>(x, g, b, y, rows, c, eps, s);
+    else launch_cta_rows<1024>(x, g, b, y, rows, c, eps, s);
+  } else if (vec_ok && x != reinterpret_cast<const float*>(y)) {
+    const int grid = (int)(rows < (int64_t)sm_count() * 4 ? rows : (int64_t)sm_count() * 4);
+    layernorm_rows_streaming<OutT><<<grid, 512, 0, s>>>(x, g, b, y, rows, cols, eps);
   } else {
     const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
     layernorm_rows_generic<OutT><<<grid, 256, 0, s>>>(x, g, b, y, rows, cols, eps);

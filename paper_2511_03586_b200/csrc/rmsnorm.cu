@@ -13,7 +13,7 @@ namespace pd {
 namespace {
 
 template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA>
-__global__ void __launch_bounds__(THREADS_PER_CTA)
+__global__ void __launch_bounds__(THREADS_PER_CTA, THREADS_PER_CTA >= 1024 ? 1 : 1024 / THREADS_PER_CTA)  // at most 64 registers: 1024 threads resident per SM
 rmsnorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__ gamma, float* __restrict__ y,
                           int64_t rows, int cols, float eps) {
   constexpr int ROWS_PER_CTA = THREADS_PER_CTA / THREADS_PER_ROW;
@@ -90,11 +90,12 @@ pd_status launch_rmsnorm(const float* x, const float* g, float* y, int64_t rows,
     else if (c <= 256) launch_warp_rows<2>(x, g, y, rows, c, eps, s);
     else if (c <= 512) launch_warp_rows<4>(x, g, y, rows, c, eps, s);
     else launch_warp_rows<8>(x, g, y, rows, c, eps, s);
-  } else if (vec_ok && cols <= 16384) {
+  } else if (vec_ok && cols <= 32768) {
     if (c <= 2048) launch_cta_rows<64>(x, g, y, rows, c, eps, s);
     else if (c <= 4096) launch_cta_rows<128>(x, g, y, rows, c, eps, s);
     else if (c <= 8192) launch_cta_rows<256>(x, g, y, rows, c, eps, s);
-    else launch_cta_rows<512>(x, g, y, rows, c, eps, s);
+    else if (c <= 16384) launch_cta_rows<512>(x, g, y, rows, c, eps, s);
+    else launch_cta_rows<1024>(x, g, y, rows, c, eps, s);
   } else {
     const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
     rmsnorm_rows_generic<<<grid, 256, 0, s>>>(x, g, y, rows, cols, eps);

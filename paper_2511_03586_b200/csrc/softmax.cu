@@ -6,8 +6,9 @@
 // global memory exactly once into registers with 128-bit loads, reduced with
 // warp shuffles, and written once.
 //   * cols <= 1024            : one warp per row (up to 8 float4 per lane)
-//   * cols <= 16384           : one CTA of 64 to 512 threads per row (8 float4 per thread)
-//   * anything else / ragged  : one CTA per row, three passes from global/L2
+//   * cols <= 32768           : one CTA of 64 to 1024 threads per row (8 float4 per thread)
+//   * longer, 16-byte aligned : one CTA per row, online (max, sum) pass from HBM, normalising pass from L2
+//   * anything else / ragged  : one CTA per row, three scalar passes from global/L2
 #include "pd_common.cuh"
 
 namespace pd {
@@ -19,7 +20,7 @@ namespace {
 // consecutive lanes.  THREADS_PER_ROW == 32: one warp per row, several rows per
 // CTA.  THREADS_PER_ROW == blockDim.x: one row per CTA.
 template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA, typename OutT>
-__global__ void __launch_bounds__(THREADS_PER_CTA)
+__global__ void __launch_bounds__(THREADS_PER_CTA, THREADS_PER_CTA >= 1024 ? 1 : 1024 / THREADS_PER_CTA)  // at most 64 registers: 1024 threads resident per SM
 softmax_rows_in_registers(const float* __restrict__ x, OutT* __restrict__ y, int64_t rows, int cols) {
   constexpr int ROWS_PER_CTA = THREADS_PER_CTA / THREADS_PER_ROW;
   constexpr int NWARPS = THREADS_PER_ROW / 32;
@@ -82,6 +83,39 @@ softmax_rows_generic(const float* __restrict__ x, OutT* __restrict__ y, int64_t 
   }
 }
 
+// Rows too long for registers (cols > 32768), 16-byte aligned: one CTA of 512 threads per row, two passes.
+// Pass 1 streams the row from HBM with 128-bit loads and keeps an online (max, sum) pair per thread (the sum is
+// rescaled whenever the running max grows), merged across the CTA; pass 2 re-reads the row, by then in L2,
+// and writes exp(x - max) / sum.
+template <typename OutT>
+__global__ void __launch_bounds__(512)
+softmax_rows_streaming(const float* __restrict__ x, OutT* __restrict__ y, int64_t rows, int64_t cols) {
+  __shared__ float scratch[2][16];
+  const int64_t cols4 = cols >> 2;
+  for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+    const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
+    float m = kNegInf, s = 0.f;
+    for (int64_t c = threadIdx.x; c < cols4; c += 512) {
+      const float4 v = __ldg(xr + c);
+      const float m4 = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+      if (m4 > m) {
+        s *= expf(m - m4);  // exp(-inf) = 0 on the first visit
+        m = m4;
+      }
+      s += (expf(v.x - m) + expf(v.y - m)) + (expf(v.z - m) + expf(v.w - m));
+    }
+    const float M = block_reduce<16, true>(m, scratch, 0);
+    s = (m == kNegInf) ? 0.f : s * expf(m - M);
+    const float inv = 1.0f / block_reduce<16, false>(s, scratch, 1);
+    for (int64_t c = threadIdx.x; c < cols4; c += 512) {
+      const float4 v = __ldg(xr + c);
+      store_out4(y, row * cols4 + c,
+                 make_float4(expf(v.x - M) * inv, expf(v.y - M) * inv, expf(v.z - M) * inv, expf(v.w - M) * inv));
+    }
+    __syncthreads();
+  }
+}
+
 template <int VPT, typename OutT>
 void launch_warp_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStream_t s) {
   constexpr int kThreads = 256, kRowsPerCta = kThreads / 32;
@@ -110,12 +144,16 @@ pd_status dispatch(const float* x, OutT* y, int64_t rows, int64_t cols, cudaStre
     else if (c <= 256) launch_warp_rows<2>(x, y, rows, c, s);
     else if (c <= 512) launch_warp_rows<4>(x, y, rows, c, s);
     else launch_warp_rows<8>(x, y, rows, c, s);
-  } else if (vec_ok && cols <= 16384) {
+  } else if (vec_ok && cols <= 32768) {
     const int c = (int)cols;
     if (c <= 2048) launch_cta_rows<64>(x, y, rows, c, s);
     else if (c <= 4096) launch_cta_rows<128>(x, y, rows, c, s);
     else if (c <= 8192) launch_cta_rows<256>(x, y, rows, c, s);
-    else launch_cta_rows<512>(x, y, rows, c, s);
+    else if (c <= 16384) launch_cta_rows<512>(x, y, rows, c, s);
+    else launch_cta_rows<1024>(x, y, rows, c, s);
+  } else if (vec_ok && x != reinterpret_cast<const float*>(y)) {
+    const int grid = (int)(rows < (int64_t)sm_count() * 4 ? rows : (int64_t)sm_count() * 4);
+    softmax_rows_streaming<OutT><<<grid, 512, 0, s>>>(x, y, rows, cols);
   } else {
     const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
     softmax_rows_generic<OutT><<<grid, 256, 0, s>>>(x, y, rows, cols);
