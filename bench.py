@@ -447,7 +447,8 @@ def run_pd(args):
         "clocks": clocks.summary(),
         "e2e": {"value": world * flops / e2e_ms / 1e9, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": x_host.numel() * 2, "d2h_bytes_per_step": y_host.numel() * 2},
-        "gpu_launches": len(stage_names) * args.steps,
+        "gpu_launches": api.pd_encoder_layer_kernel_count(shape.batch, shape.seq, shape.hidden, shape.heads,
+                                                          shape.ffn) * args.steps,
         "device_timeout_code": timeout_code,
         "stages_ms": stages,
         "roofline": roofline,

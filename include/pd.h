@@ -122,6 +122,25 @@ pd_status pd_gemm_bf16(const void* A, const void* B, void* C, int64_t M, int64_t
  * concurrent launches.  Other values: PD_ERR_BAD_SHAPE. */
 pd_status pd_set_gemm_tile_mode(int mode);
 
+/* Contraction with a LayerNorm epilogue: operators "matmul"/"bmm", "add" and
+ * "layernorm" of the paper's table "ML operators optimized using PerfLLM" as
+ * one kernel (its Section on fusing operators motivates keeping intermediates
+ * out of memory):
+ *   S[m, :] = A[m, :] B + bias + residual[m, :]              (fp32)
+ *   Y[m, :] = (S[m, :] - mean_m) / sqrt(var_m + eps) * gamma + beta
+ * with mean_m and the biased variance var_m taken over the N columns of row m.
+ * A: bf16 [M, K]; B: bf16 [K, N]; bias: fp32 [N] or NULL; residual: bf16 [M, N]
+ * or NULL; gamma, beta: fp32 [N]; Y: bf16 [M, N]; all row-major, contiguous,
+ * device pointers, 16-byte aligned, K a multiple of 8 (else PD_ERR_ALIGNMENT).
+ * N must be a multiple of 256 and at most 2048 (the N / 256 CTAs holding one
+ * row block form a thread-block cluster and exchange row statistics through
+ * distributed shared memory), else PD_ERR_UNSUPPORTED.  The caller owns every
+ * buffer; Y must not overlap an input.  M = 0 is a no-op.  Accumulation, the
+ * sum S and the statistics are fp32; only Y is rounded to bf16. */
+pd_status pd_gemm_bias_residual_layernorm(const void* A, const void* B, const float* bias, const void* residual,
+                                          const float* gamma, const float* beta, void* Y, int64_t M, int64_t N,
+                                          int64_t K, float eps, cudaStream_t stream);
+
 /* Fused multi-head scaled-dot-product attention (operators "bmm", "softmax",
  * "bmm" of the paper's table chained per head; scores and probabilities stay
  * on the SM).  qkv: bf16 [batch*seq, 3*heads*64] = column blocks [Q | K | V],
@@ -174,6 +193,21 @@ pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, const pd_encod
                                const void* x, void* y, void* workspace, size_t workspace_bytes,
                                cudaStream_t stream);
 
+/* Tuning and testing aid for the layer entry points (no counterpart in the
+ * paper, whose table lists "layernorm" as an operator of its own).  mode 0
+ * (default): when hidden is a multiple of 256 and at most 2048, each of the two
+ * LayerNorms runs inside the epilogue of the contraction that feeds it (the
+ * CTAs that hold one row block's column tiles form a thread-block cluster and
+ * exchange per-row means and centred second moments through distributed shared
+ * memory), so the fp32 pre-LayerNorm tensor is never written; other hidden sizes use the separate row kernel.
+ * mode 1: always the separate row kernel (the contraction writes the fp32 sum
+ * to the workspace).  Both forms compute the statistics in fp32 from the same
+ * fp32 sums and differ only in summation order.  The mode also decides how much
+ * workspace pd_encoder_layer_workspace_bytes reports: set it before asking.
+ * Process-wide, not thread-safe against concurrent calls.  Other values:
+ * PD_ERR_BAD_SHAPE. */
+pd_status pd_set_layernorm_fusion(int mode);
+
 /* Allocation-free variant of pd_encoder_layer_fwd (the paper has no counterpart:
  * this entry point exists for integration reasons only).  Some callers cannot
  * obtain device memory at the point where they need a layer: a serving process
@@ -186,8 +220,8 @@ pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, const pd_encod
  *  - Same arguments, results and error codes as pd_encoder_layer_fwd, minus the
  *    workspace.  A shape whose intermediates need more than the array holds
  *    (pd_encoder_layer_workspace_bytes(desc) > 32 MiB; BERT-large fits up to
- *    about 1400 tokens) is rejected with PD_ERR_WORKSPACE_TOO_SMALL and nothing
- *    is enqueued.
+ *    about 1800 tokens, 1400 with the LayerNorms unfused) is rejected with
+ *    PD_ERR_WORKSPACE_TOO_SMALL and nothing is enqueued.
  *  - The call allocates nothing: no cudaMalloc/cudaFree and no allocating
  *    library routine, on any call.
  *  - The first call on each device looks up the array's device address
@@ -207,8 +241,15 @@ pd_status pd_encoder_layer_fwd_static(const pd_encoder_layer_desc* desc, const p
  * call WAITS for the layer to finish and writes the device time of stage i, in
  * milliseconds, to stage_ms[i] (host pointer, pd_encoder_layer_stage_count()
  * floats).  pd_encoder_layer_stage_name(i) names stage i (static storage, ""
- * when out of range).  Results in y are identical to pd_encoder_layer_fwd. */
+ * when out of range).  Results in y are identical to pd_encoder_layer_fwd.
+ * A LayerNorm that runs inside its contraction's epilogue is timed with that
+ * contraction, and its own stage reports (nearly) zero. */
 int pd_encoder_layer_stage_count(void);
+/* Number of kernels one pd_encoder_layer_fwd call enqueues for `desc` under the
+ * current fusion mode (0 for an invalid, unsupported or empty desc): five for
+ * BERT-large (QKV GEMM, attention, output projection + LayerNorm, FFN up + GELU,
+ * FFN down + LayerNorm). */
+int pd_encoder_layer_kernel_count(const pd_encoder_layer_desc* desc);
 const char* pd_encoder_layer_stage_name(int stage);
 pd_status pd_encoder_layer_fwd_profiled(const pd_encoder_layer_desc* desc,
                                         const pd_encoder_layer_weights* weights, const void* x, void* y,

@@ -65,6 +65,9 @@ def _load() -> ctypes.CDLL:
                                  i64, i64, i64, i64, vp]
     lib.pd_gemm_bf16.restype = st
     lib.pd_set_gemm_tile_mode.argtypes = [ctypes.c_int]; lib.pd_set_gemm_tile_mode.restype = st
+    lib.pd_set_layernorm_fusion.argtypes = [ctypes.c_int]; lib.pd_set_layernorm_fusion.restype = st
+    lib.pd_gemm_bias_residual_layernorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_float, vp]
+    lib.pd_gemm_bias_residual_layernorm.restype = st
     lib.pd_attention_fwd.argtypes = [vp, vp, i64, i64, i64, vp]; lib.pd_attention_fwd.restype = st
     lib.pd_encoder_layer_workspace_bytes.argtypes = [ctypes.POINTER(EncoderLayerDesc)]
     lib.pd_encoder_layer_workspace_bytes.restype = ctypes.c_size_t
@@ -76,6 +79,8 @@ def _load() -> ctypes.CDLL:
     lib.pd_encoder_layer_fwd_static.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.POINTER(EncoderLayerWeights),
                                                 vp, vp, vp]
     lib.pd_encoder_layer_fwd_static.restype = st
+    lib.pd_encoder_layer_kernel_count.argtypes = [ctypes.POINTER(EncoderLayerDesc)]
+    lib.pd_encoder_layer_kernel_count.restype = ctypes.c_int
     lib.pd_encoder_layer_stage_count.argtypes = []; lib.pd_encoder_layer_stage_count.restype = ctypes.c_int
     lib.pd_encoder_layer_stage_name.argtypes = [ctypes.c_int]
     lib.pd_encoder_layer_stage_name.restype = ctypes.c_char_p
@@ -176,6 +181,27 @@ def pd_gemm_bf16_raw(a_ptr, b_ptr, c_ptr, M, N, K, lda, ldb, ldc, b_is_nk, c_dty
                              strideA, strideB, strideC, _stream(stream))
 
 
+def pd_set_layernorm_fusion(mode: int) -> None:
+    """0: LayerNorm inside the feeding contraction's epilogue where the shape allows; 1: separate row kernel."""
+    _check(_lib.pd_set_layernorm_fusion(int(mode)), "pd_set_layernorm_fusion")
+
+
+def pd_gemm_bias_residual_layernorm(a, b, bias, residual, gamma, beta, eps: float, y=None, stream=None) -> torch.Tensor:
+    """Y = LayerNorm(A @ B + bias + residual) for bf16 A [M,K], B [K,N], residual [M,N] (or None),
+    fp32 bias (or None), gamma, beta [N]; bf16 Y."""
+    M, K = a.shape
+    N = b.shape[1]
+    if y is None:
+        y = torch.empty(M, N, dtype=torch.bfloat16, device=a.device)
+    _check(_lib.pd_gemm_bias_residual_layernorm(
+        _dev(a, torch.bfloat16, "a"), _dev(b, torch.bfloat16, "b"),
+        None if bias is None else _dev(bias, torch.float32, "bias"),
+        None if residual is None else _dev(residual, torch.bfloat16, "residual"),
+        _dev(gamma, torch.float32, "gamma"), _dev(beta, torch.float32, "beta"), _dev(y, torch.bfloat16, "y"),
+        M, N, K, float(eps), _stream(stream)), "pd_gemm_bias_residual_layernorm")
+    return y
+
+
 def pd_attention_fwd(qkv: torch.Tensor, *, batch: int, seq: int, heads: int, ctx: torch.Tensor | None = None,
                      stream=None) -> torch.Tensor:
     """qkv bf16 [batch*seq, 3*heads*64] -> ctx bf16 [batch*seq, heads*64]."""
@@ -257,6 +283,11 @@ def pd_encoder_layer_fwd_static(params: EncoderLayerParams, x: torch.Tensor, y: 
                                             _dev(y, torch.bfloat16, "y"), _stream(stream)),
            "pd_encoder_layer_fwd_static")
     return y
+
+
+def pd_encoder_layer_kernel_count(batch: int, seq: int, hidden: int, heads: int, ffn: int) -> int:
+    d = EncoderLayerDesc(batch, seq, hidden, heads, ffn, 1e-5)
+    return int(_lib.pd_encoder_layer_kernel_count(ctypes.byref(d)))
 
 
 def pd_encoder_layer_stage_names() -> list[str]:

@@ -4,11 +4,11 @@
 //   QKV = X Wqkv + bqkv                                   (GEMM, bias epilogue)
 //   Ctx = softmax(Q K^T / 8) V  per (batch, head)         (fused attention kernel for seq <= 512;
 //                                                          otherwise batched GEMM, softmax, batched GEMM)
-//   pre = Ctx Wo + bo + X                                 (GEMM, bias + residual epilogue, fp32)
-//   H1  = LayerNorm(pre)                                  (row kernel, bf16 out)
+//   H1  = LayerNorm(Ctx Wo + bo + X)                      (GEMM with bias + residual + LayerNorm epilogue)
 //   Mid = GELU(H1 W1 + b1)                                (GEMM, bias + GELU epilogue)
-//   pre = Mid W2 + b2 + H1                                (GEMM, bias + residual epilogue, fp32)
-//   Y   = LayerNorm(pre)                                  (row kernel, bf16 out)
+//   Y   = LayerNorm(Mid W2 + b2 + H1)                     (GEMM with bias + residual + LayerNorm epilogue)
+// When the hidden size does not suit the fused LayerNorm epilogue (or it is switched off), the two
+// LayerNorm GEMMs write their fp32 sum to a scratch tensor and the LayerNorm row kernel follows.
 #include "pd_common.cuh"
 
 namespace pd {
@@ -37,6 +37,15 @@ bool supported_desc(const pd_encoder_layer_desc* d) {
 
 bool use_fused_attention(const pd_encoder_layer_desc* d) { return fused_attention_supported(d->seq, kHeadDim); }
 
+int g_layernorm_fusion = 0;  // 0: fuse LayerNorm into the GEMM where the shape allows, 1: always separate kernels
+
+bool use_fused_layernorm(const pd_encoder_layer_desc* d) {
+  if (g_layernorm_fusion == 1) return false;
+  GemmProblem g;
+  g.M = (int64_t)d->batch * d->seq; g.N = d->hidden; g.K = d->hidden;
+  return gemm_layernorm_supported(g);
+}
+
 Workspace plan(const pd_encoder_layer_desc* d) {
   const size_t T = (size_t)d->batch * d->seq, H = d->hidden, F = d->ffn, S = d->seq;
   // scores and probabilities are materialised only on the unfused attention path
@@ -47,7 +56,8 @@ Workspace plan(const pd_encoder_layer_desc* d) {
   w.scores = off; off += round_up(score_elems * 4);
   w.probs = off; off += round_up(score_elems * 2);
   w.ctx = off; off += round_up(T * H * 2);
-  w.pre = off; off += round_up(T * H * 4);
+  // fp32 pre-LayerNorm sums: not materialised when the LayerNorm runs inside the GEMM
+  w.pre = off; off += round_up(use_fused_layernorm(d) ? 0 : T * H * 4);
   w.h1 = off; off += round_up(T * H * 2);
   w.mid = off; off += round_up(T * F * 2);
   w.total = off;
@@ -139,15 +149,24 @@ pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_we
       if ((st = launch_gemm(g, stream)) != PD_OK) return st;
     }
   }
+  const bool fuse_ln = use_fused_layernorm(desc);
   mark();
-  {  // output projection + bias + residual (fp32 sum kept for the LayerNorm)
+  {  // output projection + bias + residual, then LayerNorm (in the epilogue, or from the fp32 sum)
     GemmProblem g;
-    g.A = ctx; g.B = w->w_o; g.C = pre; g.M = T; g.N = H; g.K = H; g.lda = H; g.ldb = H; g.ldc = H;
-    g.c_dtype = PD_F32; g.bias = w->b_o; g.residual = xb; g.ldr = H;
-    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+    g.A = ctx; g.B = w->w_o; g.M = T; g.N = H; g.K = H; g.lda = H; g.ldb = H; g.ldc = H;
+    g.bias = w->b_o; g.residual = xb; g.ldr = H;
+    if (fuse_ln) {
+      g.C = h1;
+      if ((st = launch_gemm_layernorm(g, w->ln1_gamma, w->ln1_beta, desc->ln_eps, stream)) != PD_OK) return st;
+      mark();
+    } else {
+      g.C = pre; g.c_dtype = PD_F32;
+      if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+      mark();
+      if ((st = launch_layernorm(pre, w->ln1_gamma, w->ln1_beta, h1, true, T, H, desc->ln_eps, stream)) != PD_OK)
+        return st;
+    }
   }
-  mark();
-  if ((st = launch_layernorm(pre, w->ln1_gamma, w->ln1_beta, h1, true, T, H, desc->ln_eps, stream)) != PD_OK) return st;
   mark();
   {  // FFN up + bias + GELU
     GemmProblem g;
@@ -156,14 +175,21 @@ pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_we
     if ((st = launch_gemm(g, stream)) != PD_OK) return st;
   }
   mark();
-  {  // FFN down + bias + residual
+  {  // FFN down + bias + residual, then LayerNorm
     GemmProblem g;
-    g.A = mid; g.B = w->w_ffn2; g.C = pre; g.M = T; g.N = H; g.K = F; g.lda = F; g.ldb = H; g.ldc = H;
-    g.c_dtype = PD_F32; g.bias = w->b_ffn2; g.residual = h1; g.ldr = H;
-    if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+    g.A = mid; g.B = w->w_ffn2; g.M = T; g.N = H; g.K = F; g.lda = F; g.ldb = H; g.ldc = H;
+    g.bias = w->b_ffn2; g.residual = h1; g.ldr = H;
+    if (fuse_ln) {
+      g.C = y;
+      st = launch_gemm_layernorm(g, w->ln2_gamma, w->ln2_beta, desc->ln_eps, stream);
+      mark();
+    } else {
+      g.C = pre; g.c_dtype = PD_F32;
+      if ((st = launch_gemm(g, stream)) != PD_OK) return st;
+      mark();
+      st = launch_layernorm(pre, w->ln2_gamma, w->ln2_beta, y, true, T, H, desc->ln_eps, stream);
+    }
   }
-  mark();
-  st = launch_layernorm(pre, w->ln2_gamma, w->ln2_beta, y, true, T, H, desc->ln_eps, stream);
   mark();
   return st;
 }
@@ -175,6 +201,17 @@ extern "C" pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, con
                                           const void* x, void* y, void* workspace, size_t workspace_bytes,
                                           cudaStream_t stream) {
   return pd::run_layer(desc, w, x, y, workspace, workspace_bytes, stream, nullptr);
+}
+
+extern "C" pd_status pd_set_layernorm_fusion(int mode) {
+  if (mode < 0 || mode > 1) return PD_ERR_BAD_SHAPE;
+  pd::g_layernorm_fusion = mode;
+  return PD_OK;
+}
+
+extern "C" int pd_encoder_layer_kernel_count(const pd_encoder_layer_desc* desc) {
+  if (!pd::valid_desc(desc) || !pd::supported_desc(desc) || desc->batch == 0) return 0;
+  return 1 + (pd::use_fused_attention(desc) ? 1 : 3) + 1 + (pd::use_fused_layernorm(desc) ? 2 : 4);
 }
 
 extern "C" int pd_encoder_layer_stage_count(void) { return pd::kStages; }

@@ -225,9 +225,10 @@ inline EncodeTiledFn encode_tiled_fn() {
 }
 
 // Tensor [outer][inner][rows][cols] of bf16 (or fp32 when `f32`) with cols
-// contiguous, 128-byte swizzle, zero fill outside the extents.  Strides in elements.
+// contiguous, 128-byte swizzle unless another is named, zero fill outside the extents.  Strides in elements.
 inline bool make_map(CUtensorMap* map, bool f32, const void* base, int64_t cols, int64_t rows, int64_t ld, int64_t n_inner,
-              int64_t stride_inner, int64_t n_outer, int64_t stride_outer, int box_cols, int box_rows) {
+              int64_t stride_inner, int64_t n_outer, int64_t stride_outer, int box_cols, int box_rows,
+              CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
   EncodeTiledFn fn = encode_tiled_fn();
   if (!fn) return false;
   const cuuint64_t esize = f32 ? 4 : 2;
@@ -241,7 +242,7 @@ inline bool make_map(CUtensorMap* map, bool f32, const void* base, int64_t cols,
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
             const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

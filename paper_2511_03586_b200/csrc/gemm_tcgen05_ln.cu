@@ -1,0 +1,486 @@
+// Y = LayerNorm(A B + bias + residual; gamma, beta): the projection, the residual
+// add and the LayerNorm that closes each half of an encoder layer in one kernel.
+//
+// LayerNorm needs whole rows, a 128 x 256 accumulator tile holds a quarter of a
+// 1024-wide row.  So the N / 256 CTAs that own the tiles of the same 128 rows
+// form a thread-block cluster and run in lockstep over the row blocks:
+//   * main loop: as in the single-CTA GEMM (TMA producer lane, MMA issuer lane,
+//     two TMEM accumulators, four 48 KiB stages);
+//   * epilogue pass 1: every epilogue thread owns one row and, with its sibling
+//     warp, the tile's 256 columns.  It forms v = acc + bias + residual in fp32,
+//     writes v back over the accumulator in tensor memory, and computes the mean
+//     and centred second moment of its 128 values (accumulated around the first
+//     value, so a large common offset costs no precision).  The sibling warps
+//     combine their two halves through shared memory;
+//   * exchange: the combined (mean, second moment) of each row goes to every CTA
+//     of the cluster with asynchronous distributed-shared-memory stores that
+//     credit the receiver's mbarrier, so nobody waits on a fence; a second
+//     cluster-wide mbarrier tells the senders that the previous tile's values
+//     have been read before they are overwritten.  Each CTA merges the N / 256
+//     partial statistics pairwise in the same fixed order;
+//   * epilogue pass 2 reads v back from tensor memory, normalises, applies gamma
+//     and beta, and stores bf16 through swizzled shared memory and TMA, while the
+//     MMA warp fills the other accumulator.
+// bias, gamma and beta of the CTA's 256 columns sit in shared memory.  The fp32
+// pre-LayerNorm tensor never exists in global memory.
+// Requirements: N a multiple of 256 and at most 2048 (cluster of up to 8 CTAs),
+// bf16 A [M, K], bf16 B [K, N], bf16 residual and output [M, N].
+// Every wait is bounded as in the other tensor-core kernels.
+#include "gemm_common.cuh"
+
+namespace pd {
+namespace {
+
+using namespace sm100;
+using namespace gemm;
+
+constexpr int BN = 256;
+constexpr int kMaxCluster = 8;
+constexpr int kStageA = BM * BK * 2, kStageB = BN * BK * 2, kStage = kStageA + kStageB;
+constexpr int kStages = 4;
+constexpr int kStagingPerWarp = 32 * 64;                        // 32 rows x 32 bf16 columns
+constexpr int kStagingBytes = kEpilogueWarps * kStagingPerWarp;
+constexpr int kStatsBytes = kMaxCluster * BM * 8;                // one (mean, M2) per source CTA and row
+constexpr int kPairBytes = BM * 8;                               // hand-over between the two warps of a row
+constexpr int kParamBytes = 3 * BN * 4;                          // bias, gamma, beta of this CTA's columns
+constexpr int kBarrierBytes = 256;
+constexpr int kSmemBytes =
+    kStages * kStage + kStagingBytes + kStatsBytes + kPairBytes + kParamBytes + kBarrierBytes + 1024;
+static_assert(kSmemBytes <= kSmemLimit, "shared memory budget");
+constexpr int kTmemCols = 2 * BN;
+
+struct LnParams {
+  const float* gamma;
+  const float* beta;
+  float eps;
+  int cluster;  // CTAs per cluster = N / 256
+};
+
+enum : int { kTimeoutLnStats = 105, kTimeoutLnPair = 106, kTimeoutLnConsumed = 107 };
+
+template <bool B_NK>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
+                                    const __grid_constant__ CUtensorMap tmap_b,
+                                    const __grid_constant__ CUtensorMap tmap_c, const KernelParams p,
+                                    const LnParams ln) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t staging_base = smem_base + kStages * kStage;
+  const uint32_t stats_base = staging_base + kStagingBytes;
+  const uint32_t pair_base = stats_base + kStatsBytes;
+  const uint32_t param_base = pair_base + kPairBytes;
+  const uint32_t bar_base = param_base + kParamBytes;
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
+  auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * kStages + a); };
+  auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * kStages + 2 + a); };
+  const uint32_t drain_bar = bar_base + 8u * (2 * kStages + 4);
+  const uint32_t stats_bar = bar_base + 8u * (2 * kStages + 5);     // this tile's statistics have all landed here
+  const uint32_t consumed_bar = bar_base + 8u * (2 * kStages + 6);  // every CTA has read the statistics sent from here
+  auto pair_bar = [&](int q) { return bar_base + 8u * (2 * kStages + 7 + q); };
+  uint8_t* ctrl = smem_gen + (bar_base - smem_base) + 8 * (2 * kStages + 11);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = (p.K + BK - 1) / BK;
+  const int nt = (int)cluster_ctarank();            // this CTA's column tile
+  const int cluster_id = blockIdx.x / ln.cluster;
+  const int num_clusters = gridDim.x / ln.cluster;  // row blocks are dealt round-robin to clusters
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(acc_full_bar(a), 1);
+      mbar_init(acc_empty_bar(a), kEpilogueThreads);
+    }
+    mbar_init(drain_bar, 1);
+    mbar_init(stats_bar, 1);                               // armed once per tile with the expected byte count
+    mbar_init(consumed_bar, ln.cluster * kEpilogueWarps);  // one arrival per epilogue warp of every CTA
+    for (int q = 0; q < 4; ++q) mbar_init(pair_bar(q), 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+    fence_proxy_async_smem();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(tmem_slot)), kTmemCols);
+    tmem_relinquish_alloc_permit();
+  }
+  tcgen05_fence_before_sync();
+  cluster_sync_all();  // every CTA's barriers exist before anyone signals them
+  tcgen05_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();
+  griddep_launch_dependents();
+
+  if (warp == 0) {
+    // ------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      prefetch_tensormap(&tmap_a);
+      prefetch_tensormap(&tmap_b);
+      uint32_t it = 0;
+      bool ok = true;
+      for (int mt = cluster_id; mt < p.tiles_m && ok; mt += num_clusters) {
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
+          const uint32_t sa = smem_base + s * kStage, sb = sa + kStageA;
+          mbar_arrive_expect_tx(full_bar(s), kStage);
+          tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, 0, 0);
+          if (B_NK) {
+            tma_load_4d(sb, &tmap_b, full_bar(s), kb * BK, nt * BN, 0, 0);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j)
+              tma_load_4d(sb + j * (64 * BK * 2), &tmap_b, full_bar(s), nt * BN + j * 64, kb * BK, 0, 0);
+          }
+        }
+      }
+      if (!ok) {
+        const uint32_t issued = it;
+        for (int s = 0; s < kStages; ++s) {
+          if ((uint32_t)s >= issued) break;
+          const uint32_t last = ((issued - 1 - s) / kStages) * kStages + s;
+          volatile int never = 0;
+          mbar_wait(full_bar(s), (last / kStages) & 1u, &never, nullptr, 0, 20000000ull);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // --------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(BM, BN, false, !B_NK);
+      uint32_t it = 0;
+      int local = 0;
+      bool ok = true;
+      for (int mt = cluster_id; mt < p.tiles_m && ok; mt += num_clusters, ++local) {
+        const int acc = local & 1;
+        const uint32_t acc_ph = (local >> 1) & 1u;
+        if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc)) { ok = false; break; }
+        tcgen05_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
+          tcgen05_fence_after_sync();
+          const uint32_t sa = smem_base + s * kStage, sb = sa + kStageA;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
+            const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
+                                         : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
+            mma_bf16_ss(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          mma_commit(empty_bar(s));
+        }
+        if (ok) mma_commit(acc_full_bar(acc));
+      }
+      if (!ok) {
+        mma_commit(drain_bar);
+        volatile int never = 0;
+        mbar_wait(drain_bar, 0, &never, nullptr, 0, 20000000ull);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int quarter = warp & 3;        // TMEM lanes 32*quarter .. +31
+    const int group = (warp - 2) >> 2;   // columns [64*(2c+group), +64), c = 0, 1; group 0 also talks to the cluster
+    const int row = quarter * 32 + lane;
+    const uint32_t buf = staging_base + (uint32_t)(warp - 2) * kStagingPerWarp;
+    const uint32_t row_addr = buf + (uint32_t)lane * 64u;
+    const uint32_t sw = (uint32_t)((lane >> 1) & 3);  // 64-byte swizzle: 16-byte unit index ^= (row / 2) % 4
+    const int n_tile = nt * BN;
+    auto col_of = [&](int i) { return ((i >> 1) * 2 + group) * 64 + (i & 1) * 32; };  // step i = 0..3
+
+    // bias, gamma and beta of this CTA's columns: shared memory copies (zeros for a missing bias)
+    {
+      const int t = threadIdx.x - 64;  // 0..255, one column each
+      float* prm = reinterpret_cast<float*>(smem_gen + (param_base - smem_base));
+      prm[t] = p.bias != nullptr ? __ldg(p.bias + n_tile + t) : 0.f;
+      prm[BN + t] = __ldg(ln.gamma + n_tile + t);
+      prm[2 * BN + t] = __ldg(ln.beta + n_tile + t);
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+    }
+
+    // The residual of this thread's row: 32 columns per step, fetched two steps ahead of their use (the first two
+    // steps of a tile while the previous tile is being stored).
+    uint4 res0[4], res1[4], res2[4];
+    auto load_residual = [&](int mt, int i, uint4 (&dst)[4]) {
+      const int m = mt * BM + row;
+      if (p.residual == nullptr || mt >= p.tiles_m || m >= p.M) return;
+      const uint4* rr = reinterpret_cast<const uint4*>(p.residual + (int64_t)m * p.ldr + n_tile + col_of(i));
+#pragma unroll
+      for (int j = 0; j < 4; ++j) dst[j] = __ldg(rr + j);
+    };
+#pragma unroll
+    for (int j = 0; j < 4; ++j) res0[j] = res1[j] = res2[j] = make_uint4(0u, 0u, 0u, 0u);
+    int local = 0;
+    if (lane == 0) prefetch_tensormap(&tmap_c);
+    load_residual(cluster_id, 0, res0);
+    load_residual(cluster_id, 1, res1);
+    for (int mt = cluster_id; mt < p.tiles_m; mt += num_clusters, ++local) {
+      const int acc = local & 1;
+      const uint32_t acc_ph = (local >> 1) & 1u;
+      const uint32_t tile_ph = local & 1u;  // phase parity of the once-per-tile barriers
+      const int m_warp = mt * BM + quarter * 32;
+      const int m = m_warp + lane;
+      // the previous tile's phase of stats_bar is complete (this warp waited for it): expect this tile's bytes
+      if (warp == 2 && lane == 0) mbar_arrive_expect_tx(stats_bar, (uint32_t)ln.cluster * BM * 8u);
+      if (!mbar_wait(acc_full_bar(acc), acc_ph, abort_flag, p.status, kTimeoutEpilogue)) break;
+      tcgen05_fence_after_sync();
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+      // ---- pass 1: v = alpha acc + bias + residual goes back into tensor memory; statistics of the 128 values
+      float shift = 0.f;
+      float a1[4] = {0.f, 0.f, 0.f, 0.f}, a2[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+      for (int i = 0; i < 4; ++i) {
+        const int c0 = col_of(i);
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(t_row + c0, r);
+        if (i + 2 < 4) load_residual(mt, i + 2, res2);
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 bv = ld_shared_v4_f32(param_base + (uint32_t)(c0 + j) * 4u);
+          r[j] = __float_as_uint(fmaf(__uint_as_float(r[j]), p.alpha, bv.x));
+          r[j + 1] = __float_as_uint(fmaf(__uint_as_float(r[j + 1]), p.alpha, bv.y));
+          r[j + 2] = __float_as_uint(fmaf(__uint_as_float(r[j + 2]), p.alpha, bv.z));
+          r[j + 3] = __float_as_uint(fmaf(__uint_as_float(r[j + 3]), p.alpha, bv.w));
+        }
+        if (p.residual != nullptr) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t w[4] = {res0[j].x, res0[j].y, res0[j].z, res0[j].w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+              r[8 * j + 2 * t] = __float_as_uint(__uint_as_float(r[8 * j + 2 * t]) + __uint_as_float(w[t] << 16));
+              r[8 * j + 2 * t + 1] =
+                  __float_as_uint(__uint_as_float(r[8 * j + 2 * t + 1]) + __uint_as_float(w[t] & 0xffff0000u));
+            }
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          res0[j] = res1[j];
+          res1[j] = res2[j];
+        }
+        tmem_st_32x32b_x32(t_row + c0, r);
+        if (i == 0) shift = __uint_as_float(r[0]);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const float d = __uint_as_float(r[j]) - shift;
+          a1[j & 3] += d;
+          a2[j & 3] = fmaf(d, d, a2[j & 3]);
+        }
+      }
+      float mean_p, m2_p;  // of this thread's 128 values
+      {
+        const float s1 = (a1[0] + a1[1]) + (a1[2] + a1[3]), s2 = (a2[0] + a2[1]) + (a2[2] + a2[3]);
+        const float mean_d = s1 * (1.0f / 128.0f);
+        mean_p = shift + mean_d;
+        m2_p = fmaxf(s2 - s1 * mean_d, 0.f);
+      }
+      // ---- the two warps of a row combine their halves; group 0 sends the result to every CTA of the cluster
+      if (group == 1) {
+        st_shared_v2_f32(pair_base + (uint32_t)row * 8u, mean_p, m2_p);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(pair_bar(quarter));
+      } else {
+        if (!mbar_wait(pair_bar(quarter), tile_ph, abort_flag, p.status, kTimeoutLnPair)) break;
+        const float2 other = ld_shared_v2_f32(pair_base + (uint32_t)row * 8u);
+        const float d = other.x - mean_p;
+        const float mean_c = fmaf(d, 0.5f, mean_p);
+        const float m2_c = m2_p + other.y + d * d * 64.0f;
+        // the values sent for the previous tile must have been read everywhere before they are overwritten
+        if (local > 0 && !mbar_wait(consumed_bar, tile_ph ^ 1u, abort_flag, p.status, kTimeoutLnConsumed)) break;
+        const uint32_t dst = stats_base + (uint32_t)(nt * BM + row) * 8u;
+#pragma unroll
+        for (int rk = 0; rk < kMaxCluster; ++rk)
+          if (rk < ln.cluster) st_async_v2_f32(map_to_cta(dst, rk), mean_c, m2_c, map_to_cta(stats_bar, rk));
+      }
+      tmem_st_wait();
+      if (!mbar_wait(stats_bar, tile_ph, abort_flag, p.status, kTimeoutLnStats)) break;
+      // ---- merge the row's partial statistics (fixed order: identical in every CTA)
+      float mean = 0.f, m2 = 0.f;
+      {
+        float2 st[kMaxCluster];
+#pragma unroll
+        for (int q = 0; q < kMaxCluster; ++q)
+          st[q] = q < ln.cluster ? ld_shared_v2_f32(stats_base + (uint32_t)(q * BM + row) * 8u) : make_float2(0.f, 0.f);
+        float cnt = 0.f;
+#pragma unroll
+        for (int q = 0; q < kMaxCluster; ++q) {
+          if (q < ln.cluster) {
+            const float tot = cnt + 256.0f;
+            const float d = st[q].x - mean;
+            m2 += st[q].y + d * d * (cnt * 256.0f / tot);
+            mean += d * (256.0f / tot);
+            cnt = tot;
+          }
+        }
+      }
+      __syncwarp();
+      if (lane < ln.cluster) mbar_arrive_cluster(map_to_cta(consumed_bar, (uint32_t)lane));
+      const float rstd = rsqrtf(m2 / (float)p.N + ln.eps);
+      load_residual(mt + num_clusters, 0, res0);  // the next tile's first residual values travel during pass 2
+      load_residual(mt + num_clusters, 1, res1);
+      if (p.residual != nullptr && mt + num_clusters < p.tiles_m && m + num_clusters * BM < p.M) {
+        const __nv_bfloat16* rr = p.residual + ((int64_t)m + (int64_t)num_clusters * BM) * p.ldr + n_tile;
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(rr + col_of(2)));  // the other two steps' lines: into L2
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(rr + col_of(3)));
+      }
+      // ---- pass 2: normalise and store, 32 columns per TMA store
+#pragma unroll 1
+      for (int i = 0; i < 4; ++i) {
+        const int c0 = col_of(i);
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(t_row + c0, r);
+        tmem_ld_wait();
+        uint32_t packed[16];
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 g = ld_shared_v4_f32(param_base + (uint32_t)(BN + c0 + j) * 4u);
+          const float4 b = ld_shared_v4_f32(param_base + (uint32_t)(2 * BN + c0 + j) * 4u);
+          const float y0 = fmaf((__uint_as_float(r[j]) - mean) * rstd, g.x, b.x);
+          const float y1 = fmaf((__uint_as_float(r[j + 1]) - mean) * rstd, g.y, b.y);
+          const float y2 = fmaf((__uint_as_float(r[j + 2]) - mean) * rstd, g.z, b.z);
+          const float y3 = fmaf((__uint_as_float(r[j + 3]) - mean) * rstd, g.w, b.w);
+          packed[j / 2] = pack_bf16(y0, y1);
+          packed[j / 2 + 1] = pack_bf16(y2, y3);
+        }
+        if (lane == 0) tma_store_wait_read<0>();  // the previous store of this warp has finished reading the buffer
+        __syncwarp();
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          st_shared_v4(row_addr + (((uint32_t)u ^ sw) << 4),
+                       make_uint4(packed[4 * u], packed[4 * u + 1], packed[4 * u + 2], packed[4 * u + 3]));
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_4d(&tmap_c, buf, n_tile + c0, m_warp, 0, 0);
+          tma_store_commit();
+        }
+      }
+      tcgen05_fence_before_sync();
+      mbar_arrive(acc_empty_bar(acc));
+    }
+    if (lane == 0) tma_store_wait_all<0>();
+    __syncwarp();
+  }
+
+  // ------------------------------------------------------------------- teardown
+  // No CTA may leave while a partner can still write its shared memory or signal its barriers.
+  __syncwarp();
+  tcgen05_fence_before_sync();
+  cluster_sync_all();
+  if (warp == 1) {
+    tcgen05_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+template <bool B_NK>
+pd_status launch_ln_variant(const GemmProblem& g, const float* gamma, const float* beta, float eps, cudaStream_t s) {
+  CUtensorMap ta, tb, tc;
+  if (!make_map(&ta, false, g.A, g.K, g.M, g.lda, 1, 0, 1, 0, BK, BM)) return PD_ERR_UNSUPPORTED;
+  const bool okb = B_NK ? make_map(&tb, false, g.B, g.K, g.N, g.ldb, 1, 0, 1, 0, BK, BN)
+                        : make_map(&tb, false, g.B, g.N, g.K, g.ldb, 1, 0, 1, 0, 64, BK);
+  if (!okb) return PD_ERR_UNSUPPORTED;
+  if (!make_map(&tc, false, g.C, g.N, g.M, g.ldc, 1, 0, 1, 0, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+    return PD_ERR_UNSUPPORTED;
+
+  KernelParams p{};
+  p.C = g.C; p.bias = g.bias; p.residual = g.residual; p.status = device_status_ptr();
+  if (!p.status) return PD_ERR_CUDA;
+  p.ldc = g.ldc; p.ldr = g.ldr;
+  p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
+  p.tiles_m = (int)((g.M + BM - 1) / BM);
+  p.tiles_n = (int)(g.N / BN);
+  p.batch_inner = 1;
+  p.num_tiles = p.tiles_m * p.tiles_n;
+  p.alpha = g.alpha; p.c_is_f32 = 0; p.gelu = 0;
+  LnParams ln{gamma, beta, eps, p.tiles_n};
+
+  auto kernel = gemm_bias_residual_layernorm_kernel<B_NK>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((sm_count() / ln.cluster) * ln.cluster);
+  cfg.blockDim = dim3(kThreads);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = ln.cluster;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  // Row blocks are dealt statically to the clusters, so launch only as many clusters as can be resident at once
+  // (a cluster has to fit inside one GPC, which can leave a few SMs without one).
+  static int resident[kMaxCluster + 1];  // per cluster size, 0 = not queried yet
+  if (resident[ln.cluster] == 0) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) {
+      (void)cudaGetLastError();
+      n = 1;
+    }
+    resident[ln.cluster] = n;
+  }
+  int clusters = resident[ln.cluster];
+  if (clusters > sm_count() / ln.cluster) clusters = sm_count() / ln.cluster;
+  if (clusters > p.tiles_m) clusters = p.tiles_m;
+  if (clusters < 1) clusters = 1;
+  cfg.gridDim = dim3(clusters * ln.cluster);
+  cudaLaunchKernelEx(&cfg, kernel, ta, tb, tc, p, ln);
+  return check_launch();
+}
+
+}  // namespace
+
+bool gemm_layernorm_supported(const GemmProblem& g) {
+  return g.N % BN == 0 && g.N / BN <= kMaxCluster && g.batch_inner == 1 && g.batch_outer == 1 && g.c_dtype == PD_BF16 &&
+         g.M >= 1 && !g.gelu;
+}
+
+pd_status launch_gemm_layernorm(const GemmProblem& g, const float* gamma, const float* beta, float eps,
+                                cudaStream_t s) {
+  if (!gemm_layernorm_supported(g)) return PD_ERR_UNSUPPORTED;
+  return g.b_is_nk ? launch_ln_variant<true>(g, gamma, beta, eps, s) : launch_ln_variant<false>(g, gamma, beta, eps, s);
+}
+
+}  // namespace pd
+
+extern "C" pd_status pd_gemm_bias_residual_layernorm(const void* A, const void* B, const float* bias,
+                                                     const void* residual, const float* gamma, const float* beta,
+                                                     void* Y, int64_t M, int64_t N, int64_t K, float eps,
+                                                     cudaStream_t stream) {
+  if (!A || !B || !gamma || !beta || !Y) return PD_ERR_NULL_POINTER;
+  if (M < 0 || N <= 0 || K <= 0 || !(eps >= 0.f)) return PD_ERR_BAD_SHAPE;
+  if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PD_ERR_BAD_SHAPE;
+  if (N % pd::BN != 0 || N / pd::BN > pd::kMaxCluster) return PD_ERR_UNSUPPORTED;
+  if (K % 8) return PD_ERR_ALIGNMENT;
+  const void* ptrs[] = {A, B, bias, residual, gamma, beta, Y};
+  for (const void* q : ptrs)
+    if (!pd::aligned16(q)) return PD_ERR_ALIGNMENT;
+  if (M == 0) return PD_OK;
+  pd_status st = pd::require_sm100();
+  if (st != PD_OK) return st;
+  pd::GemmProblem g;
+  g.A = A; g.B = B; g.C = Y; g.M = M; g.N = N; g.K = K; g.lda = K; g.ldb = N; g.ldc = N;
+  g.bias = bias; g.residual = static_cast<const __nv_bfloat16*>(residual); g.ldr = N;
+  return pd::launch_gemm_layernorm(g, gamma, beta, eps, stream);
+}

@@ -137,6 +137,12 @@ pd_status launch_gemm(const GemmProblem& p, cudaStream_t s);
 bool gemm_pair_tiles_profitable(const GemmProblem& p);
 void set_gemm_tile_mode(int mode);
 pd_status launch_gemm_pair(const GemmProblem& p, cudaStream_t s);
+// C = LayerNorm(alpha A B + bias + residual; gamma, beta, eps) over the N columns of each row, bf16 out, in one
+// kernel: the CTAs that hold the column tiles of a row block form a cluster and exchange row statistics.
+// N must be a multiple of 256, at most 2048.
+bool gemm_layernorm_supported(const GemmProblem& p);
+pd_status launch_gemm_layernorm(const GemmProblem& p, const float* gamma, const float* beta, float eps,
+                                cudaStream_t s);
 
 // Fused attention on qkv[batch*seq, 3*heads*64] -> ctx[batch*seq, heads*64] (both bf16).
 bool fused_attention_supported(int64_t seq, int64_t head_dim);

@@ -116,6 +116,21 @@ def gemm_integer_inputs(M: int, N: int, K: int, seed: int = 0, batch: int = 1,
     return {"a_bits": f32_to_bf16_bits(a), "b_bits": f32_to_bf16_bits(b), "a": a, "b": b}
 
 
+def gemm_layernorm_inputs(M: int, N: int, K: int, seed: int = 0, bias_mean: float = 0.0):
+    """Operands of a projection followed by residual add and LayerNorm: A [M, K], B [K, N] ~ N(0, 1/sqrt(K))
+    and residual [M, N] ~ N(0, 1), rounded to bf16; bias ~ N(bias_mean, 0.1), gamma ~ U(0.5, 1.5),
+    beta ~ N(0, 0.1) in fp32."""
+    rng = _rng(seed)
+    s = 1.0 / np.sqrt(K)
+    a_bits = f32_to_bf16_bits(_normal(rng, (M, K), 0.0, s))
+    b_bits = f32_to_bf16_bits(_normal(rng, (K, N), 0.0, s))
+    r_bits = f32_to_bf16_bits(_normal(rng, (M, N), 0.0, 1.0))
+    return {"a_bits": a_bits, "b_bits": b_bits, "residual_bits": r_bits,
+            "a": bf16_bits_to_f32(a_bits), "b": bf16_bits_to_f32(b_bits), "residual": bf16_bits_to_f32(r_bits),
+            "bias": _normal(rng, (N,), bias_mean, 0.1), "gamma": _uniform(rng, (N,), 0.5, 1.5),
+            "beta": _normal(rng, (N,), 0.0, 0.1), "eps": 1e-5}
+
+
 @dataclass(frozen=True)
 class EncoderLayerShape:
     batch: int = 32
