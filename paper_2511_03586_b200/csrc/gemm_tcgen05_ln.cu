@@ -6,12 +6,13 @@
 // form a thread-block cluster and run in lockstep over the row blocks:
 //   * main loop: as in the single-CTA GEMM (TMA producer lane, MMA issuer lane,
 //     two TMEM accumulators, four 48 KiB stages);
-//   * epilogue pass 1: every epilogue thread owns one row and, with its sibling
-//     warp, the tile's 256 columns.  It forms v = acc + bias + residual in fp32,
-//     writes v back over the accumulator in tensor memory, and computes the mean
-//     and centred second moment of its 128 values (accumulated around the first
-//     value, so a large common offset costs no precision).  The sibling warps
-//     combine their two halves through shared memory;
+//   * epilogue pass 1 (sixteen warps, so that four per scheduler hide each
+//     other's latencies): every epilogue thread owns 64 columns of one row.  It
+//     forms v = acc + bias + residual in fp32, writes v back over the
+//     accumulator in tensor memory, and computes the mean and centred second
+//     moment of its 64 values (accumulated around the first value, so a large
+//     common offset costs no precision).  The four warps that share a row
+//     combine their parts through shared memory;
 //   * exchange: the combined (mean, second moment) of each row goes to every CTA
 //     of the cluster with asynchronous distributed-shared-memory stores that
 //     credit the receiver's mbarrier, so nobody waits on a fence; a second
@@ -38,10 +39,14 @@ constexpr int BN = 256;
 constexpr int kMaxCluster = 8;
 constexpr int kStageA = BM * BK * 2, kStageB = BN * BK * 2, kStage = kStageA + kStageB;
 constexpr int kStages = 4;
-constexpr int kStagingPerWarp = 32 * 64;                        // 32 rows x 32 bf16 columns
-constexpr int kStagingBytes = kEpilogueWarps * kStagingPerWarp;
+constexpr int kLnEpilogueWarps = 16;                             // four per TMEM lane quarter: 64 columns each
+constexpr int kLnEpilogueThreads = 32 * kLnEpilogueWarps;
+constexpr int kLnThreads = 64 + kLnEpilogueThreads;
+constexpr int kStep = 16;                                        // columns per epilogue step
+constexpr int kStagingPerWarp = 32 * kStep * 2;                  // 32 rows x 16 bf16 columns
+constexpr int kStagingBytes = kLnEpilogueWarps * kStagingPerWarp;
 constexpr int kStatsBytes = kMaxCluster * BM * 8;                // one (mean, M2) per source CTA and row
-constexpr int kPairBytes = BM * 8;                               // hand-over between the two warps of a row
+constexpr int kPairBytes = 3 * BM * 8;                           // hand-over from the three other warps of a row
 constexpr int kParamBytes = 3 * BN * 4;                          // bias, gamma, beta of this CTA's columns
 constexpr int kBarrierBytes = 256;
 constexpr int kSmemBytes =
@@ -59,7 +64,7 @@ struct LnParams {
 enum : int { kTimeoutLnStats = 105, kTimeoutLnPair = 106, kTimeoutLnConsumed = 107 };
 
 template <bool B_NK>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kLnThreads, 1)
 gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
                                     const __grid_constant__ CUtensorMap tmap_b,
                                     const __grid_constant__ CUtensorMap tmap_c, const KernelParams p,
@@ -97,12 +102,12 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(acc_full_bar(a), 1);
-      mbar_init(acc_empty_bar(a), kEpilogueThreads);
+      mbar_init(acc_empty_bar(a), kLnEpilogueThreads);
     }
     mbar_init(drain_bar, 1);
     mbar_init(stats_bar, 1);                               // armed once per tile with the expected byte count
-    mbar_init(consumed_bar, ln.cluster * kEpilogueWarps);  // one arrival per epilogue warp of every CTA
-    for (int q = 0; q < 4; ++q) mbar_init(pair_bar(q), 1);
+    mbar_init(consumed_bar, ln.cluster * kLnEpilogueWarps);  // one arrival per epilogue warp of every CTA
+    for (int q = 0; q < 4; ++q) mbar_init(pair_bar(q), 3);
     *abort_flag = 0;
     fence_barrier_init();
     fence_proxy_async_smem();
@@ -191,64 +196,66 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
   } else {
     // ------------------------------------------------------------------ epilogue
     const int quarter = warp & 3;        // TMEM lanes 32*quarter .. +31
-    const int group = (warp - 2) >> 2;   // columns [64*(2c+group), +64), c = 0, 1; group 0 also talks to the cluster
+    const int group = (warp - 2) >> 2;   // columns [64*group, +64); group 0 also talks to the cluster
     const int row = quarter * 32 + lane;
     const uint32_t buf = staging_base + (uint32_t)(warp - 2) * kStagingPerWarp;
-    const uint32_t row_addr = buf + (uint32_t)lane * 64u;
-    const uint32_t sw = (uint32_t)((lane >> 1) & 3);  // 64-byte swizzle: 16-byte unit index ^= (row / 2) % 4
+    const uint32_t row_addr = buf + (uint32_t)lane * 32u;
+    const uint32_t sw = (uint32_t)((lane >> 2) & 1);  // 32-byte swizzle: 16-byte unit index ^= (row / 4) % 2
     const int n_tile = nt * BN;
-    auto col_of = [&](int i) { return ((i >> 1) * 2 + group) * 64 + (i & 1) * 32; };  // step i = 0..3
+    const int c_base = 64 * group;       // this thread's first column inside the tile
 
     // bias, gamma and beta of this CTA's columns: shared memory copies (zeros for a missing bias)
     {
-      const int t = threadIdx.x - 64;  // 0..255, one column each
       float* prm = reinterpret_cast<float*>(smem_gen + (param_base - smem_base));
-      prm[t] = p.bias != nullptr ? __ldg(p.bias + n_tile + t) : 0.f;
-      prm[BN + t] = __ldg(ln.gamma + n_tile + t);
-      prm[2 * BN + t] = __ldg(ln.beta + n_tile + t);
-      asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+      for (int t = threadIdx.x - 64; t < 3 * BN; t += kLnEpilogueThreads) {
+        const int c = n_tile + (t & (BN - 1));
+        prm[t] = t < BN ? (p.bias != nullptr ? __ldg(p.bias + c) : 0.f) : (t < 2 * BN ? __ldg(ln.gamma + c) : __ldg(ln.beta + c));
+      }
+      asm volatile("bar.sync 1, %0;" ::"n"(kLnEpilogueThreads) : "memory");
     }
 
-    // The residual of this thread's row: 32 columns per step, fetched two steps ahead of their use (the first two
-    // steps of a tile while the previous tile is being stored).
-    uint4 res0[4], res1[4], res2[4];
-    auto load_residual = [&](int mt, int i, uint4 (&dst)[4]) {
+    // The residual of this thread's 64 columns of one row, fetched one tile ahead of its use.
+    uint4 res[4][2];
+    auto load_residual = [&](int mt) {
       const int m = mt * BM + row;
       if (p.residual == nullptr || mt >= p.tiles_m || m >= p.M) return;
-      const uint4* rr = reinterpret_cast<const uint4*>(p.residual + (int64_t)m * p.ldr + n_tile + col_of(i));
+      const uint4* rr = reinterpret_cast<const uint4*>(p.residual + (int64_t)m * p.ldr + n_tile + c_base);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) dst[j] = __ldg(rr + j);
+      for (int i = 0; i < 4; ++i) {
+        res[i][0] = __ldg(rr + 2 * i);
+        res[i][1] = __ldg(rr + 2 * i + 1);
+      }
     };
 #pragma unroll
-    for (int j = 0; j < 4; ++j) res0[j] = res1[j] = res2[j] = make_uint4(0u, 0u, 0u, 0u);
+    for (int i = 0; i < 4; ++i) res[i][0] = res[i][1] = make_uint4(0u, 0u, 0u, 0u);
     int local = 0;
     if (lane == 0) prefetch_tensormap(&tmap_c);
-    load_residual(cluster_id, 0, res0);
-    load_residual(cluster_id, 1, res1);
+    load_residual(cluster_id);
     for (int mt = cluster_id; mt < p.tiles_m; mt += num_clusters, ++local) {
       const int acc = local & 1;
       const uint32_t acc_ph = (local >> 1) & 1u;
       const uint32_t tile_ph = local & 1u;  // phase parity of the once-per-tile barriers
       const int m_warp = mt * BM + quarter * 32;
-      const int m = m_warp + lane;
       // the previous tile's phase of stats_bar is complete (this warp waited for it): expect this tile's bytes
       if (warp == 2 && lane == 0) mbar_arrive_expect_tx(stats_bar, (uint32_t)ln.cluster * BM * 8u);
+      // the next tile's residual (one 128-byte line per thread) starts its way from DRAM into L2 a tile ahead
+      if (p.residual != nullptr && mt + num_clusters < p.tiles_m && (mt + num_clusters) * BM + row < p.M)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(p.residual + ((int64_t)(mt + num_clusters) * BM + row) * p.ldr +
+                                                      n_tile + c_base));
       if (!mbar_wait(acc_full_bar(acc), acc_ph, abort_flag, p.status, kTimeoutEpilogue)) break;
       tcgen05_fence_after_sync();
-      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-      // ---- pass 1: v = alpha acc + bias + residual goes back into tensor memory; statistics of the 128 values
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c_base;
+      // ---- pass 1: v = alpha acc + bias + residual goes back into tensor memory; statistics of the 64 values
       float shift = 0.f;
       float a1[4] = {0.f, 0.f, 0.f, 0.f}, a2[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll 1
+#pragma unroll
       for (int i = 0; i < 4; ++i) {
-        const int c0 = col_of(i);
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(t_row + c0, r);
-        if (i + 2 < 4) load_residual(mt, i + 2, res2);
+        uint32_t r[kStep];
+        tmem_ld_32x32b_x16(t_row + i * kStep, r);
         tmem_ld_wait();
 #pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          const float4 bv = ld_shared_v4_f32(param_base + (uint32_t)(c0 + j) * 4u);
+        for (int j = 0; j < kStep; j += 4) {
+          const float4 bv = ld_shared_v4_f32(param_base + (uint32_t)(c_base + i * kStep + j) * 4u);
           r[j] = __float_as_uint(fmaf(__uint_as_float(r[j]), p.alpha, bv.x));
           r[j + 1] = __float_as_uint(fmaf(__uint_as_float(r[j + 1]), p.alpha, bv.y));
           r[j + 2] = __float_as_uint(fmaf(__uint_as_float(r[j + 2]), p.alpha, bv.z));
@@ -256,8 +263,8 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
         if (p.residual != nullptr) {
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const uint32_t w[4] = {res0[j].x, res0[j].y, res0[j].z, res0[j].w};
+          for (int j = 0; j < 2; ++j) {
+            const uint32_t w[4] = {res[i][j].x, res[i][j].y, res[i][j].z, res[i][j].w};
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
               r[8 * j + 2 * t] = __float_as_uint(__uint_as_float(r[8 * j + 2 * t]) + __uint_as_float(w[t] << 16));
@@ -266,38 +273,38 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
             }
           }
         }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          res0[j] = res1[j];
-          res1[j] = res2[j];
-        }
-        tmem_st_32x32b_x32(t_row + c0, r);
+        tmem_st_32x32b_x16(t_row + i * kStep, r);
         if (i == 0) shift = __uint_as_float(r[0]);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
+        for (int j = 0; j < kStep; ++j) {
           const float d = __uint_as_float(r[j]) - shift;
           a1[j & 3] += d;
           a2[j & 3] = fmaf(d, d, a2[j & 3]);
         }
       }
-      float mean_p, m2_p;  // of this thread's 128 values
+      load_residual(mt + num_clusters);  // the next tile's residual travels during the exchange and pass 2
+      float mean_p, m2_p;  // of this thread's 64 values
       {
         const float s1 = (a1[0] + a1[1]) + (a1[2] + a1[3]), s2 = (a2[0] + a2[1]) + (a2[2] + a2[3]);
-        const float mean_d = s1 * (1.0f / 128.0f);
+        const float mean_d = s1 * (1.0f / 64.0f);
         mean_p = shift + mean_d;
         m2_p = fmaxf(s2 - s1 * mean_d, 0.f);
       }
-      // ---- the two warps of a row combine their halves; group 0 sends the result to every CTA of the cluster
-      if (group == 1) {
-        st_shared_v2_f32(pair_base + (uint32_t)row * 8u, mean_p, m2_p);
+      // ---- the four warps of a row combine their parts; group 0 sends the result to every CTA of the cluster
+      if (group != 0) {
+        st_shared_v2_f32(pair_base + (uint32_t)((group - 1) * BM + row) * 8u, mean_p, m2_p);
         __syncwarp();
         if (lane == 0) mbar_arrive(pair_bar(quarter));
       } else {
         if (!mbar_wait(pair_bar(quarter), tile_ph, abort_flag, p.status, kTimeoutLnPair)) break;
-        const float2 other = ld_shared_v2_f32(pair_base + (uint32_t)row * 8u);
-        const float d = other.x - mean_p;
-        const float mean_c = fmaf(d, 0.5f, mean_p);
-        const float m2_c = m2_p + other.y + d * d * 64.0f;
+        float mean_c = mean_p, m2_c = m2_p;
+#pragma unroll
+        for (int g = 1; g < 4; ++g) {  // counts 64 g and 64: the merge weights are g / (g + 1) and 1 / (g + 1)
+          const float2 other = ld_shared_v2_f32(pair_base + (uint32_t)((g - 1) * BM + row) * 8u);
+          const float d = other.x - mean_c;
+          m2_c += other.y + d * d * (64.0f * (float)g / (float)(g + 1));
+          mean_c = fmaf(d, 1.0f / (float)(g + 1), mean_c);
+        }
         // the values sent for the previous tile must have been read everywhere before they are overwritten
         if (local > 0 && !mbar_wait(consumed_bar, tile_ph ^ 1u, abort_flag, p.status, kTimeoutLnConsumed)) break;
         const uint32_t dst = stats_base + (uint32_t)(nt * BM + row) * 8u;
@@ -314,38 +321,28 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
 #pragma unroll
         for (int q = 0; q < kMaxCluster; ++q)
           st[q] = q < ln.cluster ? ld_shared_v2_f32(stats_base + (uint32_t)(q * BM + row) * 8u) : make_float2(0.f, 0.f);
-        float cnt = 0.f;
+        mean = st[0].x;
+        m2 = st[0].y;
 #pragma unroll
-        for (int q = 0; q < kMaxCluster; ++q) {
+        for (int q = 1; q < kMaxCluster; ++q) {  // counts 256 q and 256
           if (q < ln.cluster) {
-            const float tot = cnt + 256.0f;
             const float d = st[q].x - mean;
-            m2 += st[q].y + d * d * (cnt * 256.0f / tot);
-            mean += d * (256.0f / tot);
-            cnt = tot;
+            m2 += st[q].y + d * d * (256.0f * (float)q / (float)(q + 1));
+            mean = fmaf(d, 1.0f / (float)(q + 1), mean);
           }
         }
       }
-      __syncwarp();
-      if (lane < ln.cluster) mbar_arrive_cluster(map_to_cta(consumed_bar, (uint32_t)lane));
       const float rstd = rsqrtf(m2 / (float)p.N + ln.eps);
-      load_residual(mt + num_clusters, 0, res0);  // the next tile's first residual values travel during pass 2
-      load_residual(mt + num_clusters, 1, res1);
-      if (p.residual != nullptr && mt + num_clusters < p.tiles_m && m + num_clusters * BM < p.M) {
-        const __nv_bfloat16* rr = p.residual + ((int64_t)m + (int64_t)num_clusters * BM) * p.ldr + n_tile;
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(rr + col_of(2)));  // the other two steps' lines: into L2
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(rr + col_of(3)));
-      }
-      // ---- pass 2: normalise and store, 32 columns per TMA store
+      // ---- pass 2: normalise and store, 16 columns per TMA store
 #pragma unroll 1
       for (int i = 0; i < 4; ++i) {
-        const int c0 = col_of(i);
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(t_row + c0, r);
+        const int c0 = c_base + i * kStep;
+        uint32_t r[kStep];
+        tmem_ld_32x32b_x16(t_row + i * kStep, r);
         tmem_ld_wait();
-        uint32_t packed[16];
+        uint32_t packed[kStep / 2];
 #pragma unroll
-        for (int j = 0; j < 32; j += 4) {
+        for (int j = 0; j < kStep; j += 4) {
           const float4 g = ld_shared_v4_f32(param_base + (uint32_t)(BN + c0 + j) * 4u);
           const float4 b = ld_shared_v4_f32(param_base + (uint32_t)(2 * BN + c0 + j) * 4u);
           const float y0 = fmaf((__uint_as_float(r[j]) - mean) * rstd, g.x, b.x);
@@ -358,7 +355,7 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         if (lane == 0) tma_store_wait_read<0>();  // the previous store of this warp has finished reading the buffer
         __syncwarp();
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < 2; ++u)
           st_shared_v4(row_addr + (((uint32_t)u ^ sw) << 4),
                        make_uint4(packed[4 * u], packed[4 * u + 1], packed[4 * u + 2], packed[4 * u + 3]));
         fence_proxy_async_smem();
@@ -370,6 +367,10 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
       }
       tcgen05_fence_before_sync();
       mbar_arrive(acc_empty_bar(acc));
+      // This warp has read the tile's statistics (long ago: the cluster-scope release is slow, so it waits here,
+      // off the critical path; the senders need it only before the next tile's exchange).
+      __syncwarp();
+      if (lane < ln.cluster) mbar_arrive_cluster(map_to_cta(consumed_bar, (uint32_t)lane));
     }
     if (lane == 0) tma_store_wait_all<0>();
     __syncwarp();
@@ -393,7 +394,7 @@ pd_status launch_ln_variant(const GemmProblem& g, const float* gamma, const floa
   const bool okb = B_NK ? make_map(&tb, false, g.B, g.K, g.N, g.ldb, 1, 0, 1, 0, BK, BN)
                         : make_map(&tb, false, g.B, g.N, g.K, g.ldb, 1, 0, 1, 0, 64, BK);
   if (!okb) return PD_ERR_UNSUPPORTED;
-  if (!make_map(&tc, false, g.C, g.N, g.M, g.ldc, 1, 0, 1, 0, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+  if (!make_map(&tc, false, g.C, g.N, g.M, g.ldc, 1, 0, 1, 0, kStep, 32, CU_TENSOR_MAP_SWIZZLE_32B))
     return PD_ERR_UNSUPPORTED;
 
   KernelParams p{};
@@ -417,7 +418,7 @@ pd_status launch_ln_variant(const GemmProblem& g, const float* gamma, const floa
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((sm_count() / ln.cluster) * ln.cluster);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(kLnThreads);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];
