@@ -246,46 +246,52 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
       tcgen05_fence_after_sync();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN + c_base;
       // ---- pass 1: v = alpha acc + bias + residual goes back into tensor memory; statistics of the 64 values
+      // (two fp32 values per instruction throughout: the epilogue is bound by instruction issue)
       float shift = 0.f;
-      float a1[4] = {0.f, 0.f, 0.f, 0.f}, a2[4] = {0.f, 0.f, 0.f, 0.f};
+      uint64_t nshift2 = 0, a1[2] = {0, 0}, a2[2] = {0, 0};
+      const uint64_t alpha2 = pack_f32x2(p.alpha, p.alpha);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         uint32_t r[kStep];
         tmem_ld_32x32b_x16(t_row + i * kStep, r);
         tmem_ld_wait();
+        uint64_t v[kStep / 2];
 #pragma unroll
         for (int j = 0; j < kStep; j += 4) {
           const float4 bv = ld_shared_v4_f32(param_base + (uint32_t)(c_base + i * kStep + j) * 4u);
-          r[j] = __float_as_uint(fmaf(__uint_as_float(r[j]), p.alpha, bv.x));
-          r[j + 1] = __float_as_uint(fmaf(__uint_as_float(r[j + 1]), p.alpha, bv.y));
-          r[j + 2] = __float_as_uint(fmaf(__uint_as_float(r[j + 2]), p.alpha, bv.z));
-          r[j + 3] = __float_as_uint(fmaf(__uint_as_float(r[j + 3]), p.alpha, bv.w));
+          v[j / 2] = fma_f32x2(pack_b32x2(r[j], r[j + 1]), alpha2, pack_f32x2(bv.x, bv.y));
+          v[j / 2 + 1] = fma_f32x2(pack_b32x2(r[j + 2], r[j + 3]), alpha2, pack_f32x2(bv.z, bv.w));
         }
         if (p.residual != nullptr) {
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
             const uint32_t w[4] = {res[i][j].x, res[i][j].y, res[i][j].z, res[i][j].w};
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
-              r[8 * j + 2 * t] = __float_as_uint(__uint_as_float(r[8 * j + 2 * t]) + __uint_as_float(w[t] << 16));
-              r[8 * j + 2 * t + 1] =
-                  __float_as_uint(__uint_as_float(r[8 * j + 2 * t + 1]) + __uint_as_float(w[t] & 0xffff0000u));
-            }
+            for (int t = 0; t < 4; ++t)
+              v[4 * j + t] = add_f32x2(v[4 * j + t], pack_b32x2(w[t] << 16, w[t] & 0xffff0000u));
           }
         }
-        tmem_st_32x32b_x16(t_row + i * kStep, r);
-        if (i == 0) shift = __uint_as_float(r[0]);
 #pragma unroll
-        for (int j = 0; j < kStep; ++j) {
-          const float d = __uint_as_float(r[j]) - shift;
-          a1[j & 3] += d;
-          a2[j & 3] = fmaf(d, d, a2[j & 3]);
+        for (int j = 0; j < kStep / 2; ++j) unpack_b32x2(v[j], r[2 * j], r[2 * j + 1]);
+        tmem_st_32x32b_x16(t_row + i * kStep, r);
+        if (i == 0) {
+          shift = __uint_as_float(r[0]);
+          nshift2 = pack_f32x2(-shift, -shift);
+        }
+#pragma unroll
+        for (int j = 0; j < kStep / 2; ++j) {
+          const uint64_t d = add_f32x2(v[j], nshift2);
+          a1[j & 1] = add_f32x2(a1[j & 1], d);
+          a2[j & 1] = fma_f32x2(d, d, a2[j & 1]);
         }
       }
       load_residual(mt + num_clusters);  // the next tile's residual travels during the exchange and pass 2
       float mean_p, m2_p;  // of this thread's 64 values
       {
-        const float s1 = (a1[0] + a1[1]) + (a1[2] + a1[3]), s2 = (a2[0] + a2[1]) + (a2[2] + a2[3]);
+        float s1a, s1b, s2a, s2b;
+        unpack_f32x2(add_f32x2(a1[0], a1[1]), s1a, s1b);
+        unpack_f32x2(add_f32x2(a2[0], a2[1]), s2a, s2b);
+        const float s1 = s1a + s1b, s2 = s2a + s2b;
         const float mean_d = s1 * (1.0f / 64.0f);
         mean_p = shift + mean_d;
         m2_p = fmaxf(s2 - s1 * mean_d, 0.f);
@@ -333,6 +339,7 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         }
       }
       const float rstd = rsqrtf(m2 / (float)p.N + ln.eps);
+      const uint64_t nmean2 = pack_f32x2(-mean, -mean), rstd2 = pack_f32x2(rstd, rstd);
       // ---- pass 2: normalise and store, 16 columns per TMA store
 #pragma unroll 1
       for (int i = 0; i < 4; ++i) {
@@ -345,10 +352,11 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         for (int j = 0; j < kStep; j += 4) {
           const float4 g = ld_shared_v4_f32(param_base + (uint32_t)(BN + c0 + j) * 4u);
           const float4 b = ld_shared_v4_f32(param_base + (uint32_t)(2 * BN + c0 + j) * 4u);
-          const float y0 = fmaf((__uint_as_float(r[j]) - mean) * rstd, g.x, b.x);
-          const float y1 = fmaf((__uint_as_float(r[j + 1]) - mean) * rstd, g.y, b.y);
-          const float y2 = fmaf((__uint_as_float(r[j + 2]) - mean) * rstd, g.z, b.z);
-          const float y3 = fmaf((__uint_as_float(r[j + 3]) - mean) * rstd, g.w, b.w);
+          const uint64_t t0 = mul_f32x2(add_f32x2(pack_b32x2(r[j], r[j + 1]), nmean2), rstd2);
+          const uint64_t t1 = mul_f32x2(add_f32x2(pack_b32x2(r[j + 2], r[j + 3]), nmean2), rstd2);
+          float y0, y1, y2, y3;
+          unpack_f32x2(fma_f32x2(t0, pack_f32x2(g.x, g.y), pack_f32x2(b.x, b.y)), y0, y1);
+          unpack_f32x2(fma_f32x2(t1, pack_f32x2(g.z, g.w), pack_f32x2(b.z, b.w)), y2, y3);
           packed[j / 2] = pack_bf16(y0, y1);
           packed[j / 2 + 1] = pack_bf16(y2, y3);
         }
@@ -367,10 +375,10 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
       }
       tcgen05_fence_before_sync();
       mbar_arrive(acc_empty_bar(acc));
-      // This warp has read the tile's statistics (long ago: the cluster-scope release is slow, so it waits here,
-      // off the critical path; the senders need it only before the next tile's exchange).
+      // Every lane of this warp has read the tile's statistics: their values went into rstd long ago, so the
+      // loads have been performed and the signal needs no release fence (which would stall the warp here).
       __syncwarp();
-      if (lane < ln.cluster) mbar_arrive_cluster(map_to_cta(consumed_bar, (uint32_t)lane));
+      if (lane < ln.cluster) mbar_arrive_cluster_relaxed(map_to_cta(consumed_bar, (uint32_t)lane));
     }
     if (lane == 0) tma_store_wait_all<0>();
     __syncwarp();
