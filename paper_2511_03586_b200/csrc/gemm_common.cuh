@@ -56,6 +56,33 @@ __device__ __forceinline__ float gelu_erf(float z) {
   return z * (z < 0.0f ? q : 1.0f - q);
 }
 
+// The same function for two values at once, in the form  max(z, 0) - t * q  (equal to z * Phi(z) on both
+// sides of zero), with the polynomial and the last step evaluated as packed fp32 pairs: the epilogue that
+// applies it is bound by instruction issue.
+__device__ __forceinline__ uint64_t gelu_erf_x2(uint64_t z2) {
+  using namespace sm100;
+  float z0, z1;
+  unpack_f32x2(z2, z0, z1);
+  const float a0 = fabsf(z0), a1 = fabsf(z1);
+  const float t0 = fminf(a0, 5.0f), t1 = fminf(a1, 5.0f);
+  const uint64_t t2 = pack_f32x2(t0, t1);
+  uint64_t p2 = pack_f32x2(2.945814984e-05f, 2.945814984e-05f);
+  p2 = fma_f32x2(p2, t2, pack_f32x2(-7.087827801e-04f, -7.087827801e-04f));
+  p2 = fma_f32x2(p2, t2, pack_f32x2(7.746013990e-03f, 7.746013990e-03f));
+  p2 = fma_f32x2(p2, t2, pack_f32x2(-5.260629289e-02f, -5.260629289e-02f));
+  p2 = fma_f32x2(p2, t2, pack_f32x2(-4.596254617e-01f, -4.596254617e-01f));
+  p2 = fma_f32x2(p2, t2, pack_f32x2(-1.150867236e+00f, -1.150867236e+00f));
+  p2 = fma_f32x2(p2, t2, pack_f32x2(-1.000017644e+00f, -1.000017644e+00f));
+  float p0, p1, q0, q1;
+  unpack_f32x2(p2, p0, p1);
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(q0) : "f"(p0));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(q1) : "f"(p1));
+  q0 = a0 > 5.0f ? 0.0f : q0;
+  q1 = a1 > 5.0f ? 0.0f : q1;
+  // t (not |z|) multiplies q: equal where q is not zero, and an infinite z stays infinite instead of 0 * inf
+  return fma_f32x2(pack_f32x2(-t0, -t1), pack_f32x2(q0, q1), pack_f32x2(fmaxf(z0, 0.0f), fmaxf(z1, 0.0f)));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -140,37 +167,44 @@ __device__ __forceinline__ void epilogue_warp(const KernelParams& p, const CUten
       tmem_ld_32x32b_x32(t_row + c0, r);
       if (has_next) nxt.load(p, m, n_tile + col_of(i + 1), row_ok);
       tmem_ld_wait();
-      float v[32];
-#pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * p.alpha;
-      if (p.bias != nullptr) {
-        if (n0 + 32 <= p.N) {
+      // two fp32 values per instruction wherever the operation exists in packed form
+      uint64_t v2[16];
+      {
+        const uint64_t alpha2 = pack_f32x2(p.alpha, p.alpha);
+        if (p.bias != nullptr && n0 + 32 <= p.N) {
 #pragma unroll
           for (int j = 0; j < 32; j += 4) {
             const float4 bv = __ldg(reinterpret_cast<const float4*>(p.bias + n0 + j));
-            v[j] += bv.x; v[j + 1] += bv.y; v[j + 2] += bv.z; v[j + 3] += bv.w;
+            v2[j / 2] = fma_f32x2(pack_b32x2(r[j], r[j + 1]), alpha2, pack_f32x2(bv.x, bv.y));
+            v2[j / 2 + 1] = fma_f32x2(pack_b32x2(r[j + 2], r[j + 3]), alpha2, pack_f32x2(bv.z, bv.w));
           }
         } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (n0 + j < p.N) v[j] += __ldg(p.bias + n0 + j);
+          for (int j = 0; j < 32; j += 2) {
+            float b0 = 0.f, b1 = 0.f;
+            if (p.bias != nullptr) {
+              if (n0 + j < p.N) b0 = __ldg(p.bias + n0 + j);
+              if (n0 + j + 1 < p.N) b1 = __ldg(p.bias + n0 + j + 1);
+            }
+            v2[j / 2] = fma_f32x2(pack_b32x2(r[j], r[j + 1]), alpha2, pack_f32x2(b0, b1));
+          }
         }
       }
       if (p.gelu) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = gelu_erf(v[j]);
+        for (int j = 0; j < 16; ++j) v2[j] = gelu_erf_x2(v2[j]);
       }
       if (p.residual != nullptr) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const uint32_t w[4] = {cur.q[j].x, cur.q[j].y, cur.q[j].z, cur.q[j].w};
 #pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            v[8 * j + 2 * t] += __uint_as_float(w[t] << 16);
-            v[8 * j + 2 * t + 1] += __uint_as_float(w[t] & 0xffff0000u);
-          }
+          for (int t = 0; t < 4; ++t) v2[4 * j + t] = add_f32x2(v2[4 * j + t], pack_b32x2(w[t] << 16, w[t] & 0xffff0000u));
         }
       }
+      float v[32];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) unpack_f32x2(v2[j], v[2 * j], v[2 * j + 1]);
       if (step == 0) {
         // the previous store of this warp must have finished reading the buffer
         if (lane == 0) tma_store_wait_read<0>();
