@@ -76,6 +76,7 @@ constexpr uint32_t kTmemS = 0, kTmemO = 256, kTmemCols = 512;
 
 constexpr float kScale = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
 constexpr float kRescaleThreshold = 16.0f;               // largest exponent of 2 tolerated before m is raised
+constexpr float kRescaleSum = 65536.0f;                  // 2^16: a block sum at most this large has no such exponent
 
 struct AttnParams {
   __nv_bfloat16* ctx;  // [batch*seq, hidden]
@@ -321,11 +322,12 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         }
         // P_{g-2} V_{g-2} read the tile rewritten below: it must have completed
         if (!mbar_wait(p_empty(slot, buf), use_ph ^ 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
-        // exponentials of the block against reference `ref`: writes P, returns the row's partial sum and
-        // the largest exponent met
-        auto exp_block = [&](float ref, float& part_out, float& amax_out) {
+        // exponentials of the block against reference `ref`: writes P and returns the row's partial sum
+        // (two fp32 values per instruction where the operation exists in packed form)
+        auto exp_block = [&](float ref) {
+          uint64_t part2[2] = {0, 0};
           float part = 0.f;
-          float a4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+          const uint64_t scale2 = pack_f32x2(kScale, kScale), nref2 = pack_f32x2(-ref, -ref);
           uint32_t r[2][32];
           tmem_ld_32x32b_x32(t_s, r[0]);
 #pragma unroll
@@ -334,58 +336,78 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
             if (cc + 1 < kBlockK / 32) tmem_ld_32x32b_x32(t_s + (cc + 1) * 32, r[(cc & 1) ^ 1]);
             const uint32_t(&rr)[32] = r[cc & 1];
             const int c0 = key0 + cc * 32;
-            float e[32];
+            uint32_t pk[16];
             if (c0 + 32 <= p.seq) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const float a = fmaf(__uint_as_float(rr[i]), kScale, -ref);
-                a4[i & 3] = fmaxf(a4[i & 3], a);
-                e[i] = ex2_approx(a);
+              for (int i = 0; i < 32; i += 2) {
+                float a0, a1;
+                unpack_f32x2(fma_f32x2(pack_b32x2(rr[i], rr[i + 1]), scale2, nref2), a0, a1);
+                const float e0 = ex2_approx(a0), e1 = ex2_approx(a1);
+                part2[(i >> 1) & 1] = add_f32x2(part2[(i >> 1) & 1], pack_f32x2(e0, e1));
+                pk[i / 2] = pack_bf16x2(e0, e1);
               }
             } else {
 #pragma unroll
-              for (int i = 0; i < 32; ++i) {
-                const float a = fmaf(__uint_as_float(rr[i]), kScale, -ref);
-                const bool valid = c0 + i < p.seq;
-                if (valid) a4[i & 3] = fmaxf(a4[i & 3], a);
-                e[i] = valid ? ex2_approx(a) : 0.f;
+              for (int i = 0; i < 32; i += 2) {
+                const float a0 = fmaf(__uint_as_float(rr[i]), kScale, -ref);
+                const float a1 = fmaf(__uint_as_float(rr[i + 1]), kScale, -ref);
+                const float e0 = c0 + i < p.seq ? ex2_approx(a0) : 0.f;
+                const float e1 = c0 + i + 1 < p.seq ? ex2_approx(a1) : 0.f;
+                part += e0 + e1;
+                pk[i / 2] = pack_bf16x2(e0, e1);
               }
             }
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) part += (e[i] + e[i + 1]) + (e[i + 2] + e[i + 3]);
             // keys 32*cc .. 32*cc+31 of the block: 16-byte units 4*cc .. 4*cc+3 of the row
 #pragma unroll
             for (int u = 0; u < 4; ++u)
               st_shared_v4(p_row + (((uint32_t)(4 * cc + u) ^ sw) << 4),
-                           make_uint4(pack_bf16x2(e[8 * u], e[8 * u + 1]), pack_bf16x2(e[8 * u + 2], e[8 * u + 3]),
-                                      pack_bf16x2(e[8 * u + 4], e[8 * u + 5]), pack_bf16x2(e[8 * u + 6], e[8 * u + 7])));
+                           make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]));
           }
-          part_out = part;
-          amax_out = fmaxf(fmaxf(a4[0], a4[1]), fmaxf(a4[2], a4[3]));
+          float s0, s1;
+          unpack_f32x2(add_f32x2(part2[0], part2[1]), s0, s1);
+          return part + (s0 + s1);
         };
-        float part, amax;
-        exp_block(mk, part, amax);
-        const bool raise = amax > kRescaleThreshold;
-        if (__any_sync(0xffffffffu, raise)) {
+        // largest exponent of the block against reference `ref` (only the rare path below needs it)
+        auto block_amax = [&](float ref) {
+          float amax = -INFINITY;
+#pragma unroll 1
+          for (int cc = 0; cc < kBlockK / 32; ++cc) {
+            uint32_t rr[32];
+            tmem_ld_32x32b_x32(t_s + cc * 32, rr);
+            tmem_ld_wait();
+            const int c0 = key0 + cc * 32;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (c0 + i < p.seq) amax = fmaxf(amax, fmaf(__uint_as_float(rr[i]), kScale, -ref));
+          }
+          return amax;
+        };
+        float part = exp_block(mk);
+        // A term above 2^16 shows in the sum, so the sum alone clears the ordinary case; !(<=) also catches NaN.
+        if (__any_sync(0xffffffffu, !(part <= kRescaleSum))) {
           // rare: this block towers over the reference.  Raise the reference of the rows concerned, rescale
           // what they have accumulated, and redo the block.  Every earlier P V product of the slot has to
-          // be complete before O is touched: the latest one is the other tile's (there is one: g >= 1).
-          if (!mbar_wait(p_empty(slot, buf ^ 1), ((t - 1u) >> 1) & 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
-          tcgen05_fence_after_sync();
-          const float alpha = raise ? ex2_approx(-amax) : 1.0f;
-          if (raise) mk += amax;
-          l *= alpha;
+          // be complete before O is touched: the latest one is the other tile's (there is one when g >= 1).
+          const float amax = block_amax(mk);
+          const bool raise = amax > kRescaleThreshold;
+          if (g > 0) {
+            if (!mbar_wait(p_empty(slot, buf ^ 1), ((t - 1u) >> 1) & 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+            tcgen05_fence_after_sync();
+            const float alpha = raise ? ex2_approx(-amax) : 1.0f;
+            l *= alpha;
 #pragma unroll
-          for (int c0 = 0; c0 < kD; c0 += 32) {
-            uint32_t o[32];
-            tmem_ld_32x32b_x32(t_o + c0, o);
-            tmem_ld_wait();
+            for (int c0 = 0; c0 < kD; c0 += 32) {
+              uint32_t o[32];
+              tmem_ld_32x32b_x32(t_o + c0, o);
+              tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-            tmem_st_32x32b_x32(t_o + c0, o);
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st_32x32b_x32(t_o + c0, o);
+            }
+            tmem_st_wait();
           }
-          tmem_st_wait();
-          exp_block(mk, part, amax);
+          if (raise) mk += amax;
+          part = exp_block(mk);
         }
         l += part;
         fence_proxy_async_smem();
