@@ -122,6 +122,34 @@ pd_status pd_gemm_bf16(const void* A, const void* B, void* C, int64_t M, int64_t
  * concurrent launches.  Other values: PD_ERR_BAD_SHAPE. */
 pd_status pd_set_gemm_tile_mode(int mode);
 
+/* Contraction with the fused epilogue the encoder layer's projections use
+ * (operators "matmul", "add" and "relu" of the paper's table "ML operators
+ * optimized using PerfLLM" in one kernel; GELU is the activation of the
+ * layer's feed-forward block):
+ *   C = act(A B + bias) + residual
+ * A: bf16 [M, K]; B: bf16 [K, N]; bias: fp32 [N] or NULL; residual: bf16 [M, N]
+ * or NULL; C: bf16 or fp32 [M, N] (c_dtype); all row-major, contiguous, device
+ * pointers, 16-byte aligned, K and N multiples of 8 (else PD_ERR_ALIGNMENT).
+ * act: 0 none, 1 GELU in its erf form z Phi(z), 2 ReLU max(z, 0); other values
+ * PD_ERR_BAD_SHAPE.  Accumulation and the epilogue are fp32; the result is
+ * rounded once, to c_dtype.  M = 0 or N = 0 is a no-op.  The caller owns every
+ * buffer; C must not overlap an input. */
+pd_status pd_gemm_bias_act(const void* A, const void* B, const float* bias, const void* residual, void* C,
+                           int64_t M, int64_t N, int64_t K, int act, pd_dtype c_dtype, cudaStream_t stream);
+
+/* SwiGLU feed-forward projection (operator "swiglu", 1 x 256 x 4096 x 448, of
+ * the same table, read as 256 tokens, 4096 inputs, 448 outputs):
+ *   Y = SiLU(X Wg) * (X Wu),   SiLU(g) = g / (1 + exp(-g)),
+ * the two contractions and the element-wise product in one kernel: each
+ * accumulator tile holds the gate and the up product of the same output
+ * columns.  X: bf16 [M, K]; Wg, Wu: bf16 [K, N]; Y: bf16 [M, N]; row-major,
+ * contiguous, device pointers, 16-byte aligned, K and N multiples of 8 (else
+ * PD_ERR_ALIGNMENT).  Accumulation and the activation are fp32; Y is rounded
+ * once, to bf16.  M = 0 or N = 0 is a no-op.  The caller owns every buffer; Y
+ * must not overlap an input. */
+pd_status pd_swiglu_gemm(const void* X, const void* Wg, const void* Wu, void* Y, int64_t M, int64_t N, int64_t K,
+                         cudaStream_t stream);
+
 /* Contraction with a LayerNorm epilogue: operators "matmul"/"bmm", "add" and
  * "layernorm" of the paper's table "ML operators optimized using PerfLLM" as
  * one kernel (its Section on fusing operators motivates keeping intermediates

@@ -41,6 +41,10 @@ def _load():
         lib.oracle_rmsnorm.argtypes = [_D, _D, _D, _I64, _I64, ctypes.c_double]
         lib.oracle_rmsnorm.restype = ctypes.c_int
         lib.oracle_bias_gelu_residual.argtypes = [_D, _D, _D, _D, _I64, _I64]
+        lib.oracle_bias_relu_residual.argtypes = [_D, _D, _D, _D, _I64, _I64]
+        lib.oracle_bias_relu_residual.restype = ctypes.c_int
+        lib.oracle_swiglu.argtypes = [_D, _D, _D, _I64]
+        lib.oracle_swiglu.restype = ctypes.c_int
         lib.oracle_gemm.argtypes = [_D, _D, _D, _I64, _I64, _I64]
         lib.oracle_attention.argtypes = [_D, _D, _D, _I64, _I64, _I64, _I64]
         lib.oracle_encoder_layer.argtypes = [_I64] * 5 + [ctypes.c_double] + [_D] * 18
@@ -98,6 +102,27 @@ def bias_gelu_residual(x, bias, r=None) -> np.ndarray:
     assert r is None or r.shape == x.shape
     out = np.empty_like(x)
     _check(_load().oracle_bias_gelu_residual(_p(x), _p(bias), _p(r), _p(out), rows, cols), "oracle_bias_gelu_residual")
+    return out
+
+
+def bias_relu_residual(x, bias=None, r=None) -> np.ndarray:
+    x = _f64(x)
+    rows, cols = x.shape
+    bias = None if bias is None else _f64(bias)
+    r = None if r is None else _f64(r)
+    assert bias is None or bias.shape == (cols,)
+    assert r is None or r.shape == x.shape
+    out = np.empty_like(x)
+    _check(_load().oracle_bias_relu_residual(_p(x), _p(bias), _p(r), _p(out), rows, cols), "oracle_bias_relu_residual")
+    return out
+
+
+def swiglu(g, u) -> np.ndarray:
+    """SiLU(g) * u element by element."""
+    g, u = _f64(g), _f64(u)
+    assert g.shape == u.shape
+    out = np.empty_like(g)
+    _check(_load().oracle_swiglu(_p(g), _p(u), _p(out), g.size), "oracle_swiglu")
     return out
 
 

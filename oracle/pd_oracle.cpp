@@ -114,6 +114,27 @@ int oracle_bias_gelu_residual(const double* x, const double* bias, const double*
   return 0;
 }
 
+// out = ReLU(x + bias) + r, ReLU(z) = max(z, 0) (operator "relu" with the bias
+// and residual terms of the fused projection epilogue); bias and r may be null.
+int oracle_bias_relu_residual(const double* x, const double* bias, const double* r, double* out,
+                              int64_t rows, int64_t cols) {
+  if (!x || !out || rows < 0 || cols <= 0) return -1;
+  for (int64_t i = 0; i < rows; ++i)
+    for (int64_t j = 0; j < cols; ++j) {
+      const double z = x[i * cols + j] + (bias ? bias[j] : 0.0);
+      const double a = z > 0.0 ? z : 0.0;
+      out[i * cols + j] = r ? a + r[i * cols + j] : a;
+    }
+  return 0;
+}
+
+// Element-wise part of operator "swiglu": out = SiLU(g) * u, SiLU(g) = g / (1 + exp(-g)).
+int oracle_swiglu(const double* g, const double* u, double* out, int64_t n) {
+  if (!g || !u || !out || n < 0) return -1;
+  for (int64_t i = 0; i < n; ++i) out[i] = g[i] / (1.0 + std::exp(-g[i])) * u[i];
+  return 0;
+}
+
 // C[M,N] = A[M,K] * B[K,N] (operator "matmul").  The loops run m, k, n so that
 // B is walked along its rows; every c[m,n] still receives its K products in
 // ascending k, so the result is bit-identical to the M N K nest above.

@@ -65,6 +65,9 @@ def _load() -> ctypes.CDLL:
                                  i64, i64, i64, i64, vp]
     lib.pd_gemm_bf16.restype = st
     lib.pd_set_gemm_tile_mode.argtypes = [ctypes.c_int]; lib.pd_set_gemm_tile_mode.restype = st
+    lib.pd_gemm_bias_act.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp]
+    lib.pd_gemm_bias_act.restype = st
+    lib.pd_swiglu_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]; lib.pd_swiglu_gemm.restype = st
     lib.pd_set_layernorm_fusion.argtypes = [ctypes.c_int]; lib.pd_set_layernorm_fusion.restype = st
     lib.pd_gemm_bias_residual_layernorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_float, vp]
     lib.pd_gemm_bias_residual_layernorm.restype = st
@@ -179,6 +182,36 @@ def pd_gemm_bf16_raw(a_ptr, b_ptr, c_ptr, M, N, K, lda, ldb, ldc, b_is_nk, c_dty
     """Direct call with explicit pointers and strides; returns the status instead of raising."""
     return _lib.pd_gemm_bf16(a_ptr, b_ptr, c_ptr, M, N, K, lda, ldb, ldc, int(b_is_nk), int(c_dtype), batch,
                              strideA, strideB, strideC, _stream(stream))
+
+
+ACT_NONE, ACT_GELU, ACT_RELU = 0, 1, 2
+
+
+def pd_gemm_bias_act(a, b, bias=None, residual=None, *, act: int = ACT_NONE, c_dtype=torch.bfloat16, c=None,
+                     stream=None) -> torch.Tensor:
+    """C = act(A @ B + bias) + residual for bf16 A [M,K], B [K,N], residual [M,N]; fp32 bias [N]."""
+    M, K = a.shape
+    N = b.shape[1]
+    if c is None:
+        c = torch.empty(M, N, dtype=c_dtype, device=a.device)
+    _check(_lib.pd_gemm_bias_act(_dev(a, torch.bfloat16, "a"), _dev(b, torch.bfloat16, "b"),
+                                 None if bias is None else _dev(bias, torch.float32, "bias"),
+                                 None if residual is None else _dev(residual, torch.bfloat16, "residual"),
+                                 _dev(c, c.dtype, "c"), M, N, K, int(act),
+                                 PD_F32 if c.dtype == torch.float32 else PD_BF16, _stream(stream)), "pd_gemm_bias_act")
+    return c
+
+
+def pd_swiglu_gemm(x, wg, wu, y=None, stream=None) -> torch.Tensor:
+    """Y = SiLU(X @ Wg) * (X @ Wu) for bf16 X [M,K], Wg, Wu [K,N]; bf16 Y."""
+    M, K = x.shape
+    N = wg.shape[1]
+    if y is None:
+        y = torch.empty(M, N, dtype=torch.bfloat16, device=x.device)
+    _check(_lib.pd_swiglu_gemm(_dev(x, torch.bfloat16, "x"), _dev(wg, torch.bfloat16, "wg"),
+                               _dev(wu, torch.bfloat16, "wu"), _dev(y, torch.bfloat16, "y"), M, N, K,
+                               _stream(stream)), "pd_swiglu_gemm")
+    return y
 
 
 def pd_set_layernorm_fusion(mode: int) -> None:

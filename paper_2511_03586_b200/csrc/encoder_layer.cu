@@ -171,7 +171,7 @@ pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_we
   {  // FFN up + bias + GELU
     GemmProblem g;
     g.A = h1; g.B = w->w_ffn1; g.C = mid; g.M = T; g.N = F; g.K = H; g.lda = H; g.ldb = F; g.ldc = F;
-    g.bias = w->b_ffn1; g.gelu = true;
+    g.bias = w->b_ffn1; g.act = 1;
     if ((st = launch_gemm(g, stream)) != PD_OK) return st;
   }
   mark();

@@ -28,7 +28,7 @@ struct KernelParams {
   int M, N, K;
   int tiles_m, tiles_n, batch_inner, num_tiles;  // num_tiles = batch_outer * batch_inner * tiles_m * tiles_n
   float alpha;
-  int c_is_f32, gelu;
+  int c_is_f32, act;  // act: 0 nothing, 1 erf-form GELU, 2 ReLU
 };
 
 // Codes left in the device status word by an expired wait.
@@ -190,9 +190,16 @@ __device__ __forceinline__ void epilogue_warp(const KernelParams& p, const CUten
           }
         }
       }
-      if (p.gelu) {
+      if (p.act == 1) {
 #pragma unroll
         for (int j = 0; j < 16; ++j) v2[j] = gelu_erf_x2(v2[j]);
+      } else if (p.act == 2) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          float z0, z1;
+          unpack_f32x2(v2[j], z0, z1);
+          v2[j] = pack_f32x2(fmaxf(z0, 0.0f), fmaxf(z1, 0.0f));
+        }
       }
       if (p.residual != nullptr) {
 #pragma unroll
@@ -237,6 +244,85 @@ __device__ __forceinline__ void epilogue_warp(const KernelParams& p, const CUten
     release(acc);
   }
   // Shared memory must outlive every store that still reads it.
+  if (lane == 0) tma_store_wait_all<0>();
+  __syncwarp();
+}
+
+// Epilogue of the gated form.  The accumulator holds G = A Wg in columns [0, BN/2) and U = A Wu in columns
+// [BN/2, BN) for the same BN/2 output columns; the warp writes SiLU(G) * U = G * U / (1 + exp(-G)) as bf16.
+// The two warps of a lane group take alternate steps of 32 output columns; each step goes out through one
+// half of the warp's staging buffer (32 rows x 64 bytes, 64-byte swizzle) and its own TMA store, so that a
+// step is staged while the previous one is still being read.
+template <int BN, typename ReleaseFn>
+__device__ __forceinline__ void epilogue_warp_gated(const KernelParams& p, const CUtensorMap* tmap_c, uint32_t tmem_base,
+                                                    uint32_t epi_base, uint32_t acc_full_bar0, volatile int* abort_flag,
+                                                    int first_tile, int tile_stride, ReleaseFn release) {
+  using namespace sm100;
+  constexpr int OC = BN / 2;            // output columns per tile
+  constexpr int STEPS = OC / 64;        // steps of 32 columns per warp and tile
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int quarter = warp & 3;
+  const int group = (warp - 2) >> 2;
+  const uint32_t buf = epi_base + (uint32_t)(warp - 2) * 4096u;
+  const uint32_t sw = (uint32_t)((lane >> 1) & 3);  // 64-byte swizzle: 16-byte unit index ^= (row / 2) % 4
+  const uint64_t nlog2e2 = pack_f32x2(-1.4426950408889634f, -1.4426950408889634f), one2 = pack_f32x2(1.0f, 1.0f);
+  int local = 0;
+  uint32_t stores = 0;
+  if (lane == 0) prefetch_tensormap(tmap_c);
+  for (int tile = first_tile; tile < p.num_tiles; tile += tile_stride, ++local) {
+    const int nt = tile % p.tiles_n;
+    const int mt = tile / p.tiles_n;
+    const int acc = local & 1;
+    const uint32_t acc_ph = (local >> 1) & 1u;
+    const int m_warp = mt * BM + quarter * 32;
+    if (!mbar_wait(acc_full_bar0 + 8u * acc, acc_ph, abort_flag, p.status, kTimeoutEpilogue)) break;
+    tcgen05_fence_after_sync();
+    const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+#pragma unroll 1
+    for (int i = 0; i < STEPS; ++i) {
+      const int c0 = (2 * i + group) * 32;
+      if (nt * OC + c0 >= p.N) break;  // uniform over the warp
+      uint32_t rg[32], ru[32];
+      tmem_ld_32x32b_x32(t_row + c0, rg);
+      tmem_ld_32x32b_x32(t_row + OC + c0, ru);
+      tmem_ld_wait();
+      uint32_t packed[16];
+#pragma unroll
+      for (int j = 0; j < 32; j += 2) {
+        const uint64_t g2 = pack_b32x2(rg[j], rg[j + 1]);
+        float x0, x1;
+        unpack_f32x2(mul_f32x2(g2, nlog2e2), x0, x1);
+        float e0, e1;
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(x0));
+        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(x1));
+        float d0, d1;
+        unpack_f32x2(add_f32x2(pack_f32x2(e0, e1), one2), d0, d1);
+        float r0, r1;
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r0) : "f"(d0));
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r1) : "f"(d1));
+        // (g * sigmoid(g)) * u, in this order: g * u alone could overflow where the product with sigmoid does not
+        float y0, y1;
+        unpack_f32x2(mul_f32x2(mul_f32x2(g2, pack_f32x2(r0, r1)), pack_b32x2(ru[j], ru[j + 1])), y0, y1);
+        packed[j / 2] = pack_bf16(y0, y1);
+      }
+      const uint32_t half = buf + (stores & 1u) * 2048u;
+      if (lane == 0) tma_store_wait_read<1>();  // the store before the previous one has finished reading this half
+      __syncwarp();
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        st_shared_v4(half + (uint32_t)lane * 64u + (((uint32_t)u ^ sw) << 4),
+                     make_uint4(packed[4 * u], packed[4 * u + 1], packed[4 * u + 2], packed[4 * u + 3]));
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) {
+        tma_store_4d(tmap_c, half, nt * OC + c0, m_warp, 0, 0);
+        tma_store_commit();
+      }
+      ++stores;
+    }
+    tcgen05_fence_before_sync();
+    release(acc);
+  }
   if (lane == 0) tma_store_wait_all<0>();
   __syncwarp();
 }

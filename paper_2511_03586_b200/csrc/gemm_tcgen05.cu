@@ -45,10 +45,14 @@ struct Cfg {
   static constexpr int kTmemCols = 2 * BN;  // two accumulators; 128, 256 or 512: a power of two
 };
 
-template <int BN, bool B_NK, bool C_F32>
+// GATED: the tile's B operand is BN/2 columns of the first weight followed by the same BN/2 columns of a
+// second one (tmap_b2), and the epilogue writes SiLU(first product) * second product, BN/2 columns wide.
+template <int BN, bool B_NK, bool C_F32, bool GATED>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                         const __grid_constant__ CUtensorMap tmap_c, const KernelParams p) {
+                         const __grid_constant__ CUtensorMap tmap_b2, const __grid_constant__ CUtensorMap tmap_c,
+                         const KernelParams p) {
+  static_assert(!GATED || (!B_NK && !C_F32 && BN >= 128), "gated form: B as [K, N], bf16 out, 64-column boxes");
   using C = Cfg<BN>;
   constexpr int kStages = C::kStages;
   extern __shared__ uint8_t smem_raw[];
@@ -100,6 +104,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     if (lane == 0) {
       prefetch_tensormap(&tmap_a);
       prefetch_tensormap(&tmap_b);
+      if (GATED) prefetch_tensormap(&tmap_b2);
       uint32_t it = 0;  // k-blocks issued so far, over all tiles
       bool ok = true;
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
@@ -114,7 +119,12 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
           const uint32_t sa = smem_base + s * C::kStage, sb = sa + C::kStageA;
           mbar_arrive_expect_tx(full_bar(s), C::kStage);
           tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, bi, bo);
-          if (B_NK) {
+          if constexpr (GATED) {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j)
+              tma_load_4d(sb + j * (64 * BK * 2), j < BN / 128 ? &tmap_b : &tmap_b2, full_bar(s),
+                          nt * (BN / 2) + (j % (BN / 128)) * 64, kb * BK, 0, 0);
+          } else if (B_NK) {
             tma_load_4d(sb, &tmap_b, full_bar(s), kb * BK, nt * BN, bi, bo);
           } else {
 #pragma unroll
@@ -173,9 +183,13 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    epilogue_warp<BN, C_F32>(
-        p, &tmap_c, tmem_base, epi_base, acc_full_bar(0), abort_flag, blockIdx.x, gridDim.x,
-        [](int mt) { return mt * BM; }, [&](int acc) { mbar_arrive(acc_empty_bar(acc)); });
+    if constexpr (GATED)
+      epilogue_warp_gated<BN>(p, &tmap_c, tmem_base, epi_base, acc_full_bar(0), abort_flag, blockIdx.x, gridDim.x,
+                              [&](int acc) { mbar_arrive(acc_empty_bar(acc)); });
+    else
+      epilogue_warp<BN, C_F32>(
+          p, &tmap_c, tmem_base, epi_base, acc_full_bar(0), abort_flag, blockIdx.x, gridDim.x,
+          [](int mt) { return mt * BM; }, [&](int acc) { mbar_arrive(acc_empty_bar(acc)); });
   }
 
   // ------------------------------------------------------------------- teardown
@@ -188,10 +202,11 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   }
 }
 
-template <int BN, bool B_NK, bool C_F32>
+template <int BN, bool B_NK, bool C_F32, bool GATED = false>
 pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
   using C = Cfg<BN>;
-  CUtensorMap ta, tb, tc;
+  constexpr int OC = GATED ? BN / 2 : BN;  // output columns per tile
+  CUtensorMap ta, tb, tb2, tc;
   if (!make_map(&ta, false, g.A, g.K, g.M, g.lda, g.batch_inner, g.strideA_inner, g.batch_outer, g.strideA_outer, BK, BM))
     return PD_ERR_UNSUPPORTED;
   const bool okb = B_NK ? make_map(&tb, false, g.B, g.K, g.N, g.ldb, g.batch_inner, g.strideB_inner, g.batch_outer,
@@ -199,10 +214,14 @@ pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
                         : make_map(&tb, false, g.B, g.N, g.K, g.ldb, g.batch_inner, g.strideB_inner, g.batch_outer,
                                    g.strideB_outer, 64, BK);
   if (!okb) return PD_ERR_UNSUPPORTED;
-  // C is written in boxes of 32 rows x 128 bytes (one epilogue warp, one chunk).
-  if (!make_map(&tc, C_F32, g.C, g.N, g.M, g.ldc, g.batch_inner, g.strideC_inner, g.batch_outer, g.strideC_outer,
-                C_F32 ? 32 : 64, 32))
-    return PD_ERR_UNSUPPORTED;
+  tb2 = tb;
+  if (GATED && !make_map(&tb2, false, g.B2, g.N, g.K, g.ldb, 1, 0, 1, 0, 64, BK)) return PD_ERR_UNSUPPORTED;
+  // C is written in boxes of 32 rows x 128 bytes (one epilogue warp, one chunk); the gated epilogue writes
+  // boxes of 32 rows x 64 bytes.
+  const bool okc = GATED ? make_map(&tc, false, g.C, g.N, g.M, g.ldc, 1, 0, 1, 0, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)
+                         : make_map(&tc, C_F32, g.C, g.N, g.M, g.ldc, g.batch_inner, g.strideC_inner, g.batch_outer,
+                                    g.strideC_outer, C_F32 ? 32 : 64, 32);
+  if (!okc) return PD_ERR_UNSUPPORTED;
 
   KernelParams p{};
   p.C = g.C; p.bias = g.bias; p.residual = g.residual; p.status = device_status_ptr();
@@ -210,14 +229,14 @@ pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
   p.ldc = g.ldc; p.strideC_inner = g.strideC_inner; p.strideC_outer = g.strideC_outer; p.ldr = g.ldr;
   p.M = (int)g.M; p.N = (int)g.N; p.K = (int)g.K;
   p.tiles_m = (int)((g.M + BM - 1) / BM);
-  p.tiles_n = (int)((g.N + BN - 1) / BN);
+  p.tiles_n = (int)((g.N + OC - 1) / OC);
   p.batch_inner = (int)g.batch_inner;
   const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n * g.batch_inner * g.batch_outer;
   if (tiles > 0x7fffffff) return PD_ERR_BAD_SHAPE;
   p.num_tiles = (int)tiles;
-  p.alpha = g.alpha; p.c_is_f32 = g.c_dtype == PD_F32; p.gelu = g.gelu;
+  p.alpha = g.alpha; p.c_is_f32 = g.c_dtype == PD_F32; p.act = g.act;
 
-  auto kernel = gemm_bf16_tcgen05_kernel<BN, B_NK, C_F32>;
+  auto kernel = gemm_bf16_tcgen05_kernel<BN, B_NK, C_F32, GATED>;
   static bool attr_set = false;  // per template instantiation
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
@@ -225,7 +244,7 @@ pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
     attr_set = true;
   }
   const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
-  launch_pdl(kernel, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, tc, p);
+  launch_pdl(kernel, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, tb2, tc, p);
   return check_launch();
 }
 
@@ -244,6 +263,15 @@ int g_tile_mode = 0;  // 0: automatic, 1: single-CTA tiles only, 2: CTA-pair til
 void set_gemm_tile_mode(int mode) { g_tile_mode = mode; }
 
 pd_status launch_gemm(const GemmProblem& g, cudaStream_t s) {
+  if (g.B2 != nullptr) {
+    // gated form: 128 x 128 output tiles, or 128 x 64 when those fill the SMs' last wave better
+    if (g.b_is_nk || g.c_dtype != PD_BF16 || g.batch_inner != 1 || g.batch_outer != 1 || g.bias || g.residual || g.act)
+      return PD_ERR_UNSUPPORTED;
+    const int64_t tiles_m = (g.M + BM - 1) / BM, sms = sm_count();
+    const int64_t t128 = tiles_m * ((g.N + 127) / 128), t64 = tiles_m * ((g.N + 63) / 64);
+    const double c128 = (double)((t128 + sms - 1) / sms) * 256.0, c64 = (double)((t64 + sms - 1) / sms) * 128.0 / 0.66;
+    return c64 < c128 ? launch_variant<128, false, false, true>(g, s) : launch_variant<256, false, false, true>(g, s);
+  }
   if (g_tile_mode == 2 || (g_tile_mode == 0 && gemm_pair_tiles_profitable(g))) return launch_gemm_pair(g, s);
   // 128 x 256 tiles reuse operands best (the 128 x 128 main loop runs at about
   // two thirds of their rate); narrower tiles are used when N is small or when
@@ -298,4 +326,39 @@ extern "C" pd_status pd_set_gemm_tile_mode(int mode) {
   if (mode < 0 || mode > 2) return PD_ERR_BAD_SHAPE;
   pd::set_gemm_tile_mode(mode);
   return PD_OK;
+}
+
+extern "C" pd_status pd_gemm_bias_act(const void* A, const void* B, const float* bias, const void* residual, void* C,
+                                      int64_t M, int64_t N, int64_t K, int act, pd_dtype c_dtype,
+                                      cudaStream_t stream) {
+  if (!A || !B || !C) return PD_ERR_NULL_POINTER;
+  if (M < 0 || N < 0 || K <= 0 || act < 0 || act > 2) return PD_ERR_BAD_SHAPE;
+  if (c_dtype != PD_BF16 && c_dtype != PD_F32) return PD_ERR_BAD_SHAPE;
+  if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PD_ERR_BAD_SHAPE;
+  if (!pd::aligned16(A) || !pd::aligned16(B) || !pd::aligned16(C) || !pd::aligned16(bias) || !pd::aligned16(residual) ||
+      K % 8 || N % 8)
+    return PD_ERR_ALIGNMENT;
+  if (M == 0 || N == 0) return PD_OK;
+  pd_status st = pd::require_sm100();
+  if (st != PD_OK) return st;
+  pd::GemmProblem g;
+  g.A = A; g.B = B; g.C = C; g.M = M; g.N = N; g.K = K; g.lda = K; g.ldb = N; g.ldc = N;
+  g.c_dtype = c_dtype; g.bias = bias; g.act = act;
+  g.residual = static_cast<const __nv_bfloat16*>(residual); g.ldr = N;
+  return pd::launch_gemm(g, stream);
+}
+
+extern "C" pd_status pd_swiglu_gemm(const void* X, const void* Wg, const void* Wu, void* Y, int64_t M, int64_t N,
+                                    int64_t K, cudaStream_t stream) {
+  if (!X || !Wg || !Wu || !Y) return PD_ERR_NULL_POINTER;
+  if (M < 0 || N < 0 || K <= 0) return PD_ERR_BAD_SHAPE;
+  if (M > 0x7fffffff || N > 0x7fffffff || K > 0x7fffffff) return PD_ERR_BAD_SHAPE;
+  if (!pd::aligned16(X) || !pd::aligned16(Wg) || !pd::aligned16(Wu) || !pd::aligned16(Y) || K % 8 || N % 8)
+    return PD_ERR_ALIGNMENT;
+  if (M == 0 || N == 0) return PD_OK;
+  pd_status st = pd::require_sm100();
+  if (st != PD_OK) return st;
+  pd::GemmProblem g;
+  g.A = X; g.B = Wg; g.B2 = Wu; g.C = Y; g.M = M; g.N = N; g.K = K; g.lda = K; g.ldb = N; g.ldc = N;
+  return pd::launch_gemm(g, stream);
 }

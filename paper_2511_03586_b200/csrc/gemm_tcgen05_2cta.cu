@@ -212,7 +212,7 @@ pd_status launch_pair_variant(const GemmProblem& g, cudaStream_t s) {
   const int64_t tiles = (int64_t)p.tiles_m * p.tiles_n * g.batch_inner * g.batch_outer;
   if (tiles > 0x7fffffff) return PD_ERR_BAD_SHAPE;
   p.num_tiles = (int)tiles;
-  p.alpha = g.alpha; p.c_is_f32 = C_F32; p.gelu = g.gelu;
+  p.alpha = g.alpha; p.c_is_f32 = C_F32; p.act = g.act;
 
   auto kernel = gemm_bf16_tcgen05_pair_kernel<B_NK, C_F32>;
   static bool attr_set = false;

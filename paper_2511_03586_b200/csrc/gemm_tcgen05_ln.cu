@@ -414,7 +414,7 @@ pd_status launch_ln_variant(const GemmProblem& g, const float* gamma, const floa
   p.tiles_n = (int)(g.N / BN);
   p.batch_inner = 1;
   p.num_tiles = p.tiles_m * p.tiles_n;
-  p.alpha = g.alpha; p.c_is_f32 = 0; p.gelu = 0;
+  p.alpha = g.alpha; p.c_is_f32 = 0; p.act = 0;
   LnParams ln{gamma, beta, eps, p.tiles_n};
 
   auto kernel = gemm_bias_residual_layernorm_kernel<B_NK>;
@@ -462,7 +462,7 @@ pd_status launch_ln_variant(const GemmProblem& g, const float* gamma, const floa
 
 bool gemm_layernorm_supported(const GemmProblem& g) {
   return g.N % BN == 0 && g.N / BN <= kMaxCluster && g.batch_inner == 1 && g.batch_outer == 1 && g.c_dtype == PD_BF16 &&
-         g.M >= 1 && !g.gelu;
+         g.M >= 1 && g.act == 0 && g.B2 == nullptr;
 }
 
 pd_status launch_gemm_layernorm(const GemmProblem& g, const float* gamma, const float* beta, float eps,

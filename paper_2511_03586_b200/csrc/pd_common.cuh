@@ -114,6 +114,7 @@ pd_status launch_bias_gelu_residual(const float* x, const float* bias, const flo
 // One (optionally batched) bf16 contraction with a fused epilogue:
 //   C[bo][bi][m,n] = epilogue(alpha * sum_k A[bo][bi][m,k] * B[bo][bi][k,n])
 //   epilogue(v)    = act(v + bias[n]) + residual[m,n]
+// or, in gated form (B2 set), with G = A B and U = A B2:  C = SiLU(G) * U  (no bias, activation or residual).
 // The batch index has two levels (outer, inner) so that the per-head operands
 // of attention can be addressed inside the packed [tokens, 3*hidden] tensor.
 struct GemmProblem {
@@ -128,7 +129,8 @@ struct GemmProblem {
   int64_t strideC_inner = 0, strideC_outer = 0;
   float alpha = 1.0f;
   const float* bias = nullptr;               // fp32 [N] or null
-  bool gelu = false;                         // erf-form GELU after the bias
+  int act = 0;                               // after the bias: 0 nothing, 1 erf-form GELU, 2 ReLU
+  const void* B2 = nullptr;                  // bf16 [K, N], row stride ldb: second weight of the gated form, or null
   const __nv_bfloat16* residual = nullptr;   // bf16 [M, N], row stride ldr, or null (unbatched only)
   int64_t ldr = 0;
 };

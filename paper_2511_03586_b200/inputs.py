@@ -131,6 +131,17 @@ def gemm_layernorm_inputs(M: int, N: int, K: int, seed: int = 0, bias_mean: floa
             "beta": _normal(rng, (N,), 0.0, 0.1), "eps": 1e-5}
 
 
+def swiglu_inputs(M: int, N: int, K: int, seed: int = 0):
+    """Operands of a SwiGLU projection: X [M, K] ~ N(0, 1), gate and up weights [K, N] ~ N(0, 1/sqrt(K)),
+    all rounded to bf16 (bit patterns and their exact float32 widenings)."""
+    rng = _rng(seed)
+    x_bits = f32_to_bf16_bits(_normal(rng, (M, K), 0.0, 1.0))
+    wg_bits = f32_to_bf16_bits(_normal(rng, (K, N), 0.0, 1.0 / np.sqrt(K)))
+    wu_bits = f32_to_bf16_bits(_normal(rng, (K, N), 0.0, 1.0 / np.sqrt(K)))
+    return {"x_bits": x_bits, "wg_bits": wg_bits, "wu_bits": wu_bits, "x": bf16_bits_to_f32(x_bits),
+            "wg": bf16_bits_to_f32(wg_bits), "wu": bf16_bits_to_f32(wu_bits)}
+
+
 @dataclass(frozen=True)
 class EncoderLayerShape:
     batch: int = 32

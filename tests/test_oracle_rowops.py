@@ -1,4 +1,4 @@
-"""Pins for the CPU oracle's row operators (softmax, layernorm, bias+GELU+residual).
+"""Pins for the CPU oracle's row operators (softmax, layernorm, rmsnorm, bias+GELU+residual, ReLU, SwiGLU).
 
 Nothing here touches the CUDA path.  Every expected value comes from a closed
 form, an invariant, an independent series or a textbook table, never from the
@@ -229,6 +229,62 @@ def test_bias_broadcast_residual_and_permutation():
 
 
 # ------------------------------------------------- library cross-check (torch f64)
+# ------------------------------------------------------------ relu, swiglu
+def test_relu_epilogue_special_cases():
+    x = np.array([[-2.0, -0.0, 0.0, 3.5], [1e-300, -1e-300, 7.0, -7.0]])
+    out = oracle.bias_relu_residual(x)
+    assert np.array_equal(out, np.array([[0.0, 0.0, 0.0, 3.5], [1e-300, 0.0, 7.0, 0.0]]))
+    # relu(z) - relu(-z) = z and relu(z) + relu(-z) = |z|
+    rng = np.random.default_rng(41)
+    z = rng.normal(size=(5, 9))
+    assert np.array_equal(oracle.bias_relu_residual(z) - oracle.bias_relu_residual(-z), z)
+    assert np.array_equal(oracle.bias_relu_residual(z) + oracle.bias_relu_residual(-z), np.abs(z))
+    # the bias is added before the kink (broadcast over rows), the residual after it
+    bias = rng.normal(size=9)
+    r = rng.normal(size=(5, 9))
+    got = oracle.bias_relu_residual(z, bias, r)
+    for i in range(5):
+        for j in range(9):
+            t = z[i, j] + bias[j]
+            assert got[i, j] == (t if t > 0 else 0.0) + r[i, j]
+    # a large negative bias switches everything off and leaves the residual
+    assert np.array_equal(oracle.bias_relu_residual(z, np.full(9, -100.0), r), r)
+
+
+def test_swiglu_closed_forms():
+    # SiLU(0) = 0; SiLU(ln 3) = ln 3 * 3/4; SiLU(-ln 3) = -ln 3 / 4
+    g = np.array([0.0, math.log(3.0), -math.log(3.0)])
+    np.testing.assert_allclose(oracle.swiglu(g, np.ones(3)), [0.0, 0.75 * math.log(3.0), -0.25 * math.log(3.0)],
+                               rtol=1e-15, atol=0)
+    rng = np.random.default_rng(42)
+    g, u = rng.normal(0, 3, size=200), rng.normal(size=200)
+    s = oracle.swiglu(g, np.ones_like(g))
+    # SiLU(g) - SiLU(-g) = g  and  SiLU(g) + SiLU(-g) = g tanh(g / 2)
+    sm = oracle.swiglu(-g, np.ones_like(g))
+    np.testing.assert_allclose(s - sm, g, rtol=1e-14, atol=1e-15)
+    np.testing.assert_allclose(s + sm, g * np.tanh(g / 2), rtol=1e-13, atol=1e-15)
+    # linear in u, and the gate is the FIRST argument: swapping the operands changes the result
+    np.testing.assert_allclose(oracle.swiglu(g, u), s * u, rtol=1e-15, atol=0)
+    assert not np.allclose(oracle.swiglu(g, u), oracle.swiglu(u, g))
+    # limits: SiLU(g) -> g for large g, -> 0 from below for very negative g; minimum value about -0.27846 at g = -1.27846
+    np.testing.assert_allclose(oracle.swiglu(np.array([40.0]), np.ones(1)), [40.0], rtol=1e-15)
+    assert -1e-15 < oracle.swiglu(np.array([-40.0]), np.ones(1))[0] < 0
+    grid = np.linspace(-3, 0, 300001)
+    vals = oracle.swiglu(grid, np.ones_like(grid))
+    assert abs(vals.min() + 0.27846454276107) < 1e-10 and abs(grid[vals.argmin()] + 1.27846454276107) < 1e-4
+
+
+def test_relu_swiglu_against_torch_float64():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(43)
+    g, u = rng.normal(0, 2, size=(7, 33)), rng.normal(size=(7, 33))
+    ref = (torch.nn.functional.silu(torch.from_numpy(g)) * torch.from_numpy(u)).numpy()
+    np.testing.assert_allclose(oracle.swiglu(g, u), ref, rtol=1e-14, atol=1e-16)
+    bias, r = rng.normal(size=33), rng.normal(size=(7, 33))
+    ref = (torch.relu(torch.from_numpy(g) + torch.from_numpy(bias)) + torch.from_numpy(r)).numpy()
+    assert np.array_equal(oracle.bias_relu_residual(g, bias, r), ref)
+
+
 def test_rowops_against_torch_float64():
     torch = pytest.importorskip("torch")
     rng = np.random.default_rng(8)
