@@ -276,6 +276,53 @@ def ops_suite(torch, api, peaks, only: str = ""):
         rowop_entry(f"bias_gelu_residual_{rows}x{cols}", ms, rows * cols * 12 + cols * 4, "configured shape")
         del xs, rs, os_, p
 
+    def bf16_rand(*shape, scale=1.0):
+        return (torch.randn(*shape, device="cuda") * scale).to(torch.bfloat16)
+
+    def gemm_entry(name, ms, flops, note):
+        tf = flops / ms / 1e9
+        out[name] = {"ms": ms, "TFLOP/s": tf, "frac_measured_sustained": tf / peaks["bf16_tflops_sustained"],
+                     "frac_nominal": tf / NOMINAL_BF16_TFLOPS, "note": note}
+
+    # small problems of the paper's operator table: less than one wave of tiles, bound by latency, not by the tensor pipe
+    M, N, K = 768, 1024, 1024
+    if wanted(f"gemm_{M}x{N}x{K}"):
+        a, b = bf16_rand(M, K), bf16_rand(K, N, scale=K ** -0.5)
+        c = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+        ms = time_launches(torch, lambda i: api.pd_gemm_bf16(a, b, c), 200)
+        gemm_entry(f"gemm_{M}x{N}x{K}_cbf16", ms, 2.0 * M * N * K, "paper shape (matmul); operands L2-resident")
+    B_, M, K, N = 192, 256, 128, 256
+    if wanted(f"bmm_{B_}x{M}x{K}x{N}"):
+        a, b = bf16_rand(B_, M, K), bf16_rand(B_, K, N, scale=K ** -0.5)
+        c = torch.empty(B_, M, N, dtype=torch.bfloat16, device="cuda")
+        ms = time_launches(torch, lambda i: api.pd_gemm_bf16(a, b, c), 200)
+        gemm_entry(f"bmm_{B_}x{M}x{K}x{N}_cbf16", ms, 2.0 * B_ * M * N * K, "paper shape (bmm); operands L2-resident")
+    M, N, K = 256, 448, 4096
+    if wanted(f"swiglu_{M}x{N}x{K}"):
+        x, wg, wu = bf16_rand(M, K), bf16_rand(K, N, scale=K ** -0.5), bf16_rand(K, N, scale=K ** -0.5)
+        y = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+        ms = time_launches(torch, lambda i: api.pd_swiglu_gemm(x, wg, wu, y), 200)
+        gemm_entry(f"swiglu_{M}x{N}x{K}", ms, 4.0 * M * N * K, "paper shape (swiglu: gate and up products + SiLU * up)")
+    M, N, K = 16384, 1024, 1024
+    if wanted(f"gemm_layernorm_{M}x{N}x{K}"):
+        as_ = [bf16_rand(M, K) for _ in range(3)]
+        rs = [bf16_rand(M, N) for _ in range(3)]
+        ys = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+        b = bf16_rand(K, N, scale=K ** -0.5)
+        bias, gam, bet = torch.randn(N, device="cuda"), torch.rand(N, device="cuda") + 0.5, torch.randn(N, device="cuda")
+        ms = time_launches(torch, lambda i: api.pd_gemm_bias_residual_layernorm(as_[i % 3], b, bias, rs[i % 3], gam, bet,
+                                                                                 1e-5, y=ys[i % 3]), 50)
+        gemm_entry(f"gemm_layernorm_{M}x{N}x{K}", ms, 2.0 * M * N * K, "the layer's output projection + residual + LayerNorm")
+        del as_, rs, ys
+    M, N, K = 16384, 4096, 1024
+    if wanted(f"gemm_bias_gelu_{M}x{N}x{K}"):
+        as_ = [bf16_rand(M, K) for _ in range(3)]
+        cs = [torch.empty(M, N, dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+        b, bias = bf16_rand(K, N, scale=K ** -0.5), torch.randn(N, device="cuda")
+        ms = time_launches(torch, lambda i: api.pd_gemm_bias_act(as_[i % 3], b, bias, None, act=api.ACT_GELU, c=cs[i % 3]), 30)
+        gemm_entry(f"gemm_bias_gelu_{M}x{N}x{K}", ms, 2.0 * M * N * K, "the layer's FFN-up projection + bias + GELU")
+        del as_, cs
+
     M, K, N = 16384, 1024, 4096
     if not wanted(f"gemm_{M}x{N}x{K}"):
         return out

@@ -169,6 +169,17 @@ pd_status pd_gemm_bias_residual_layernorm(const void* A, const void* B, const fl
                                           const float* gamma, const float* beta, void* Y, int64_t M, int64_t N,
                                           int64_t K, float eps, cudaStream_t stream);
 
+/* Tuning and testing aid (no counterpart in the paper).  mode 0 (default): a
+ * contraction with K >= 2048 whose output tiles would cover less than half of
+ * the SMs (the paper's swiglu 256 x 448 x 4096 is such a problem) is split
+ * along K over a thread-block cluster of 2, 4 or 8 CTAs
+ * that add their partial sums through distributed shared memory before the
+ * epilogue; results differ from the unsplit kernels only by fp32 summation
+ * order.  mode 1: never split.  Splitting applies only under
+ * pd_set_gemm_tile_mode(0).  Process-wide, not thread-safe against concurrent
+ * launches.  Other values: PD_ERR_BAD_SHAPE. */
+pd_status pd_set_gemm_split_k(int mode);
+
 /* Fused multi-head scaled-dot-product attention (operators "bmm", "softmax",
  * "bmm" of the paper's table chained per head; scores and probabilities stay
  * on the SM).  qkv: bf16 [batch*seq, 3*heads*64] = column blocks [Q | K | V],

@@ -68,6 +68,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_gemm_bias_act.argtypes = [vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_int, ctypes.c_int, vp]
     lib.pd_gemm_bias_act.restype = st
     lib.pd_swiglu_gemm.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp]; lib.pd_swiglu_gemm.restype = st
+    lib.pd_set_gemm_split_k.argtypes = [ctypes.c_int]; lib.pd_set_gemm_split_k.restype = st
     lib.pd_set_layernorm_fusion.argtypes = [ctypes.c_int]; lib.pd_set_layernorm_fusion.restype = st
     lib.pd_gemm_bias_residual_layernorm.argtypes = [vp, vp, vp, vp, vp, vp, vp, i64, i64, i64, ctypes.c_float, vp]
     lib.pd_gemm_bias_residual_layernorm.restype = st
@@ -212,6 +213,11 @@ def pd_swiglu_gemm(x, wg, wu, y=None, stream=None) -> torch.Tensor:
                                _dev(wu, torch.bfloat16, "wu"), _dev(y, torch.bfloat16, "y"), M, N, K,
                                _stream(stream)), "pd_swiglu_gemm")
     return y
+
+
+def pd_set_gemm_split_k(mode: int) -> None:
+    """0: split K over a thread-block cluster when a contraction has few output tiles; 1: never."""
+    _check(_lib.pd_set_gemm_split_k(int(mode)), "pd_set_gemm_split_k")
 
 
 def pd_set_layernorm_fusion(mode: int) -> None:

@@ -261,8 +261,16 @@ namespace {
 int g_tile_mode = 0;  // 0: automatic, 1: single-CTA tiles only, 2: CTA-pair tiles whenever the shape allows
 }
 void set_gemm_tile_mode(int mode) { g_tile_mode = mode; }
+namespace {
+int g_split_k_mode = 0;  // 0: split K over a cluster when the problem has few tiles, 1: never
+}
+void set_gemm_split_k_mode(int mode) { g_split_k_mode = mode; }
 
 pd_status launch_gemm(const GemmProblem& g, cudaStream_t s) {
+  if (g_tile_mode == 0 && g_split_k_mode != 1) {
+    const int split = gemm_split_k_factor(g);
+    if (split > 0 && (g.B2 == nullptr || (!g.bias && !g.residual && !g.act))) return launch_gemm_split_k(g, split, s);
+  }
   if (g.B2 != nullptr) {
     // gated form: 128 x 128 output tiles, or 128 x 64 when those fill the SMs' last wave better
     if (g.b_is_nk || g.c_dtype != PD_BF16 || g.batch_inner != 1 || g.batch_outer != 1 || g.bias || g.residual || g.act)
@@ -361,4 +369,10 @@ extern "C" pd_status pd_swiglu_gemm(const void* X, const void* Wg, const void* W
   pd::GemmProblem g;
   g.A = X; g.B = Wg; g.B2 = Wu; g.C = Y; g.M = M; g.N = N; g.K = K; g.lda = K; g.ldb = N; g.ldc = N;
   return pd::launch_gemm(g, stream);
+}
+
+extern "C" pd_status pd_set_gemm_split_k(int mode) {
+  if (mode < 0 || mode > 1) return PD_ERR_BAD_SHAPE;
+  pd::set_gemm_split_k_mode(mode);
+  return PD_OK;
 }

@@ -138,7 +138,12 @@ pd_status launch_gemm(const GemmProblem& p, cudaStream_t s);
 // The same contraction on 256 x 256 tiles computed by pairs of CTAs (cta_group::2).
 bool gemm_pair_tiles_profitable(const GemmProblem& p);
 void set_gemm_tile_mode(int mode);
+void set_gemm_split_k_mode(int mode);
 pd_status launch_gemm_pair(const GemmProblem& p, cudaStream_t s);
+// Split-K over a thread-block cluster for problems with few output tiles: the cluster size to use (0: none) and
+// the launcher (128 x 256 accumulator tiles, reduce-scatter through distributed shared memory).
+int gemm_split_k_factor(const GemmProblem& p);
+pd_status launch_gemm_split_k(const GemmProblem& p, int split, cudaStream_t s);
 // C = LayerNorm(alpha A B + bias + residual; gamma, beta, eps) over the N columns of each row, bf16 out, in one
 // kernel: the CTAs that hold the column tiles of a row block form a cluster and exchange row statistics.
 // N must be a multiple of 256, at most 2048.

@@ -118,6 +118,30 @@ def test_swiglu_gate_and_up_are_not_swapped_and_saturate(api):
     assert np.isfinite(y2).all() and np.all(y2[x < 0] == 0) and np.array_equal(y2[x > 0], 128.0 * x[x > 0] ** 2)
 
 
+@pytest.mark.parametrize("shape", [(768, 1024, 2048), (127, 248, 3000), (64, 64, 4096), (1100, 1032, 2048), (512, 264, 8192)])
+def test_split_k_over_a_cluster_matches_the_unsplit_kernel(api, shape):
+    # few output tiles: under automatic tiles K is split over a cluster of 2, 4 or 8 CTAs; forced off, one CTA per tile
+    M, N, K = shape
+    p = inputs.gemm_layernorm_inputs(M, N, K, seed=K)
+    a, b, bias, r = dev_bf16(p["a_bits"]), dev_bf16(p["b_bits"]), dev_f32(p["bias"]), dev_bf16(p["residual_bits"])
+    ref = _oracle_bias_act(p, 1, True, True)
+    outs = []
+    for mode in (0, 1):
+        api.pd_set_gemm_split_k(mode)
+        try:
+            c = Guarded((M, N), torch.float32)
+            api.pd_gemm_bias_act(a, b, bias, r, act=1, c=c.t)
+            torch.cuda.synchronize()
+            c.check()
+            c2 = api.pd_gemm_bias_act(a, b, bias, r, act=1, c_dtype=torch.float32)
+            assert torch.equal(c.t, c2)                     # repeatable
+            outs.append(host(c.t))
+            assert max_rel_floored(outs[-1], ref) < TOL_F32
+        finally:
+            api.pd_set_gemm_split_k(0)
+    assert max_rel_floored(outs[0], outs[1]) < 1e-5
+
+
 def test_argument_errors(api):
     from paper_2511_03586_b200.api import PdError
     a = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
