@@ -232,6 +232,22 @@ pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, const pd_encod
                                const void* x, void* y, void* workspace, size_t workspace_bytes,
                                cudaStream_t stream);
 
+/* A stack of n_layers encoder layers of the same shape, each with its own
+ * weights (weights: host array of n_layers structs), layer l + 1 reading what
+ * layer l wrote (the paper's kernels come from whole models: its Section
+ * "Search with PerfLLM" evaluates operators "in existing models"):
+ *   X_0 = x,  X_{l+1} = layer_l(X_l),  y = X_{n_layers}.
+ * Every layer is pd_encoder_layer_fwd; all of them are enqueued on `stream`
+ * without host synchronisation, the activations between layers (bf16) alternate
+ * between two tensors inside the workspace.  workspace: 256-byte aligned, at
+ * least pd_encoder_stack_workspace_bytes(desc, n_layers) bytes (0 for an invalid
+ * desc or n_layers < 1), else PD_ERR_WORKSPACE_TOO_SMALL.  Other arguments and
+ * errors as for pd_encoder_layer_fwd; n_layers < 1 is PD_ERR_BAD_SHAPE. */
+size_t pd_encoder_stack_workspace_bytes(const pd_encoder_layer_desc* desc, int n_layers);
+pd_status pd_encoder_stack_fwd(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* weights,
+                               int n_layers, const void* x, void* y, void* workspace, size_t workspace_bytes,
+                               cudaStream_t stream);
+
 /* Tuning and testing aid for the layer entry points (no counterpart in the
  * paper, whose table lists "layernorm" as an operator of its own).  mode 0
  * (default): when hidden is a multiple of 256 and at most 2048, each of the two

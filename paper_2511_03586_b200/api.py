@@ -78,6 +78,11 @@ def _load() -> ctypes.CDLL:
     lib.pd_encoder_layer_fwd.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.POINTER(EncoderLayerWeights),
                                          vp, vp, vp, ctypes.c_size_t, vp]
     lib.pd_encoder_layer_fwd.restype = st
+    lib.pd_encoder_stack_workspace_bytes.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.c_int]
+    lib.pd_encoder_stack_workspace_bytes.restype = ctypes.c_size_t
+    lib.pd_encoder_stack_fwd.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.POINTER(EncoderLayerWeights),
+                                         ctypes.c_int, vp, vp, vp, ctypes.c_size_t, vp]
+    lib.pd_encoder_stack_fwd.restype = st
     lib.pd_encoder_layer_static_scratch_bytes.argtypes = []
     lib.pd_encoder_layer_static_scratch_bytes.restype = ctypes.c_size_t
     lib.pd_encoder_layer_fwd_static.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.POINTER(EncoderLayerWeights),
@@ -301,6 +306,25 @@ def pd_encoder_layer_fwd(params: EncoderLayerParams, x: torch.Tensor, *, batch: 
     _check(_lib.pd_encoder_layer_fwd(ctypes.byref(d), ctypes.byref(w), _dev(x, torch.bfloat16, "x"),
                                      _dev(y, torch.bfloat16, "y"), workspace.data_ptr(), workspace.numel(),
                                      _stream(stream)), "pd_encoder_layer_fwd")
+    return y
+
+
+def pd_encoder_stack_fwd(layers, x: torch.Tensor, *, batch: int, seq: int, heads: int, ln_eps: float = 1e-5,
+                         y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None):
+    """Runs ``layers`` (a list of EncoderLayerParams of one shape) one after the other on x [batch*seq, hidden]."""
+    T, hidden = x.shape
+    if T != batch * seq:
+        raise ValueError("x must be [batch*seq, hidden]")
+    d = EncoderLayerDesc(batch, seq, hidden, heads, layers[0].w_ffn1.shape[1], ln_eps)
+    if y is None:
+        y = torch.empty_like(x)
+    if workspace is None:
+        nbytes = int(_lib.pd_encoder_stack_workspace_bytes(ctypes.byref(d), len(layers)))
+        workspace = torch.empty(max(nbytes, 1), dtype=torch.uint8, device=x.device)
+    w = (EncoderLayerWeights * len(layers))(*[p.as_struct() for p in layers])
+    _check(_lib.pd_encoder_stack_fwd(ctypes.byref(d), w, len(layers), _dev(x, torch.bfloat16, "x"),
+                                     _dev(y, torch.bfloat16, "y"), workspace.data_ptr(), workspace.numel(),
+                                     _stream(stream)), "pd_encoder_stack_fwd")
     return y
 
 

@@ -203,6 +203,39 @@ extern "C" pd_status pd_encoder_layer_fwd(const pd_encoder_layer_desc* desc, con
   return pd::run_layer(desc, w, x, y, workspace, workspace_bytes, stream, nullptr);
 }
 
+// ---- a stack of layers ---------------------------------------------------------
+extern "C" size_t pd_encoder_stack_workspace_bytes(const pd_encoder_layer_desc* desc, int n_layers) {
+  if (!pd::valid_desc(desc) || !pd::supported_desc(desc) || n_layers < 1) return 0;
+  const size_t act = pd::round_up((size_t)desc->batch * desc->seq * desc->hidden * 2);
+  return pd::plan(desc).total + (n_layers > 1 ? 2 * act : 0);
+}
+
+extern "C" pd_status pd_encoder_stack_fwd(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* weights,
+                                          int n_layers, const void* x, void* y, void* workspace,
+                                          size_t workspace_bytes, cudaStream_t stream) {
+  using namespace pd;
+  if (!desc || !weights || !x || !y) return PD_ERR_NULL_POINTER;
+  if (!valid_desc(desc) || n_layers < 1) return PD_ERR_BAD_SHAPE;
+  if (!supported_desc(desc)) return PD_ERR_UNSUPPORTED;
+  if (desc->batch == 0) return PD_OK;
+  if (!workspace) return PD_ERR_NULL_POINTER;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return PD_ERR_ALIGNMENT;
+  if (workspace_bytes < pd_encoder_stack_workspace_bytes(desc, n_layers)) return PD_ERR_WORKSPACE_TOO_SMALL;
+  // layout: the layer's own workspace, then two activation tensors the layers alternate between
+  const size_t layer_bytes = plan(desc).total;
+  const size_t act = round_up((size_t)desc->batch * desc->seq * desc->hidden * 2);
+  uint8_t* base = static_cast<uint8_t*>(workspace);
+  void* pong[2] = {base + layer_bytes, base + layer_bytes + act};
+  const void* in = x;
+  for (int l = 0; l < n_layers; ++l) {
+    void* out = l == n_layers - 1 ? y : pong[l & 1];
+    const pd_status st = run_layer(desc, weights + l, in, out, workspace, layer_bytes, stream, nullptr);
+    if (st != PD_OK) return st;
+    in = out;
+  }
+  return PD_OK;
+}
+
 extern "C" pd_status pd_set_layernorm_fusion(int mode) {
   if (mode < 0 || mode > 1) return PD_ERR_BAD_SHAPE;
   pd::g_layernorm_fusion = mode;

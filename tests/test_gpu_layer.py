@@ -144,6 +144,56 @@ def test_bert_large_shape_sampled_sequences(api):
     assert float((z.var(dim=1, unbiased=False) - 1).abs().max()) < 0.05
 
 
+def test_stack_of_layers_against_oracle(api):
+    # three layers with different weights: layer l + 1 reads what layer l wrote
+    shape = inputs.EncoderLayerShape(batch=2, seq=72, hidden=256, heads=4, ffn=384)
+    ps = [inputs.encoder_layer_inputs(shape, seed=10 + l) for l in range(3)]
+    layers = [_device_params(api, p) for p in ps]
+    x = dev_bf16(ps[0]["x_bits"])
+    y = api.pd_encoder_stack_fwd(layers, x, batch=shape.batch, seq=shape.seq, heads=shape.heads)
+    ref = inputs.bf16_bits_to_f32(ps[0]["x_bits"]).astype(np.float64)
+    for p in ps:
+        q = dict(p)
+        q["x_bits"] = None
+        w = {m: inputs.bf16_bits_to_f32(p[m + "_bits"]) for m in _MATS}
+        ref = oracle.encoder_layer(ref, w["w_qkv"], p["b_qkv"], w["w_o"], p["b_o"], w["w_ffn1"], p["b_ffn1"],
+                                   w["w_ffn2"], p["b_ffn2"], p["ln1_gamma"], p["ln1_beta"], p["ln2_gamma"],
+                                   p["ln2_beta"], batch=shape.batch, seq=shape.seq, heads=shape.heads,
+                                   ln_eps=np.float32(shape.ln_eps))
+    assert max_rel_floored(host(y), ref) < TOL
+    # the same as three single-layer calls, bit for bit
+    z = x
+    for layer in layers:
+        z = api.pd_encoder_layer_fwd(layer, z, batch=shape.batch, seq=shape.seq, heads=shape.heads)
+    assert torch.equal(y, z)
+
+
+def test_layer_replays_from_a_cuda_graph(api):
+    # the whole layer is enqueued without host synchronisation, so it can be captured once and replayed
+    shape = inputs.EncoderLayerShape(batch=2, seq=136, hidden=512, heads=8, ffn=1024)
+    p = inputs.encoder_layer_inputs(shape, seed=4)
+    params = _device_params(api, p)
+    x = dev_bf16(p["x_bits"])
+    kw = dict(batch=shape.batch, seq=shape.seq, heads=shape.heads)
+    nbytes = api.pd_encoder_layer_workspace_bytes(shape.batch, shape.seq, shape.hidden, shape.heads, shape.ffn)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    y_direct = api.pd_encoder_layer_fwd(params, x, workspace=ws, **kw).clone()      # also the one-time set-up calls
+    y = torch.zeros_like(y_direct)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            api.pd_encoder_layer_fwd(params, x, y=y, workspace=ws, **kw)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        y.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(y, y_direct)
+    assert max_rel_floored(host(y), _oracle_layer(p, shape)) < TOL
+
+
 def test_layer_argument_errors(api):
     shape = inputs.EncoderLayerShape(batch=1, seq=16, hidden=64, heads=1, ffn=64)
     p = inputs.encoder_layer_inputs(shape, seed=0)
