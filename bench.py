@@ -265,6 +265,16 @@ def ops_suite(torch, api, peaks, only: str = ""):
         rowop_entry(f"rmsnorm_{rows}x{cols}", ms, rows * cols * 8 + cols * 4, "paper shape")
         del xs, ys
 
+    rows, cols = 4096, 4096
+    if wanted(f"reducemean_{rows}x{cols}"):
+        x = torch.from_numpy(inputs.rmsnorm_inputs(rows, cols)["x"]).cuda()
+        n = pool_size(rows * cols * 4)
+        xs = [x.clone() for _ in range(n)]
+        ys = [torch.empty(rows, dtype=torch.float32, device="cuda") for _ in range(n)]
+        ms = time_launches(torch, lambda i: api.pd_reducemean(xs[i % n], ys[i % n]), 60)
+        rowop_entry(f"reducemean_{rows}x{cols}", ms, rows * cols * 4 + rows * 4, "paper shape")
+        del xs, ys
+
     rows, cols = 16384, 4096
     if wanted(f"bias_gelu_residual_{rows}x{cols}"):
         p = inputs.bias_gelu_residual_inputs(rows, cols)

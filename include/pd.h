@@ -122,6 +122,14 @@ pd_status pd_gemm_bf16(const void* A, const void* B, void* C, int64_t M, int64_t
  * concurrent launches.  Other values: PD_ERR_BAD_SHAPE. */
 pd_status pd_set_gemm_tile_mode(int mode);
 
+/* Mean over the last dimension (operator "reducemean" of the paper's table,
+ * 4096 x 4096; the reduction LayerNorm's first statistic also takes):
+ *   y[i] = (1 / cols) * sum_j x[i,j].
+ * x: fp32 [rows, cols], contiguous rows; y: fp32 [rows]; device pointers, 4-byte
+ * aligned (else PD_ERR_ALIGNMENT; 16-byte aligned x with cols % 4 == 0 takes the
+ * vector path).  fp32 arithmetic, tree-shaped summation.  rows = 0 is a no-op. */
+pd_status pd_reducemean(const float* x, float* y, int64_t rows, int64_t cols, cudaStream_t stream);
+
 /* Contraction with the fused epilogue the encoder layer's projections use
  * (operators "matmul", "add" and "relu" of the paper's table "ML operators
  * optimized using PerfLLM" in one kernel; GELU is the activation of the

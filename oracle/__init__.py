@@ -41,6 +41,8 @@ def _load():
         lib.oracle_rmsnorm.argtypes = [_D, _D, _D, _I64, _I64, ctypes.c_double]
         lib.oracle_rmsnorm.restype = ctypes.c_int
         lib.oracle_bias_gelu_residual.argtypes = [_D, _D, _D, _D, _I64, _I64]
+        lib.oracle_reducemean.argtypes = [_D, _D, _I64, _I64]
+        lib.oracle_reducemean.restype = ctypes.c_int
         lib.oracle_bias_relu_residual.argtypes = [_D, _D, _D, _D, _I64, _I64]
         lib.oracle_bias_relu_residual.restype = ctypes.c_int
         lib.oracle_swiglu.argtypes = [_D, _D, _D, _I64]
@@ -91,6 +93,14 @@ def rmsnorm(x, gamma, eps: float) -> np.ndarray:
     assert gamma.shape == (cols,)
     y = np.empty_like(x)
     _check(_load().oracle_rmsnorm(_p(x), _p(gamma), _p(y), rows, cols, float(eps)), "oracle_rmsnorm")
+    return y
+
+
+def reducemean(x) -> np.ndarray:
+    x = _f64(x)
+    rows, cols = x.shape
+    y = np.empty(rows, dtype=np.float64)
+    _check(_load().oracle_reducemean(_p(x), _p(y), rows, cols), "oracle_reducemean")
     return y
 
 

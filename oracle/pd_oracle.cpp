@@ -96,6 +96,19 @@ int oracle_rmsnorm(const double* x, const double* gamma, double* y, int64_t rows
   return 0;
 }
 
+// Mean over the last dimension (operator "reducemean"):
+//   N M  y[i] += x[i,j] / M
+int oracle_reducemean(const double* x, double* y, int64_t rows, int64_t cols) {
+  if (!x || !y || rows < 0 || cols <= 0) return -1;
+  const double M = static_cast<double>(cols);
+  for (int64_t i = 0; i < rows; ++i) {
+    double acc = 0.0;
+    for (int64_t j = 0; j < cols; ++j) acc += x[i * cols + j] / M;
+    y[i] = acc;
+  }
+  return 0;
+}
+
 // GELU in its erf form.
 static double gelu_erf(double z) { return 0.5 * z * (1.0 + std::erf(z / std::sqrt(2.0))); }
 

@@ -60,6 +60,7 @@ def _load() -> ctypes.CDLL:
     lib.pd_softmax.argtypes = [vp, vp, i64, i64, vp]; lib.pd_softmax.restype = st
     lib.pd_layernorm.argtypes = [vp, vp, vp, vp, i64, i64, ctypes.c_float, vp]; lib.pd_layernorm.restype = st
     lib.pd_rmsnorm.argtypes = [vp, vp, vp, i64, i64, ctypes.c_float, vp]; lib.pd_rmsnorm.restype = st
+    lib.pd_reducemean.argtypes = [vp, vp, i64, i64, vp]; lib.pd_reducemean.restype = st
     lib.pd_bias_gelu_residual.argtypes = [vp, vp, vp, vp, i64, i64, vp]; lib.pd_bias_gelu_residual.restype = st
     lib.pd_gemm_bf16.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, ctypes.c_int, ctypes.c_int,
                                  i64, i64, i64, i64, vp]
@@ -145,6 +146,15 @@ def pd_rmsnorm(x, gamma, eps: float, y=None, stream=None) -> torch.Tensor:
         y = torch.empty_like(x)
     _check(_lib.pd_rmsnorm(_dev(x, torch.float32, "x"), _dev(gamma, torch.float32, "gamma"),
                            _dev(y, torch.float32, "y"), rows, cols, float(eps), _stream(stream)), "pd_rmsnorm")
+    return y
+
+
+def pd_reducemean(x, y=None, stream=None) -> torch.Tensor:
+    rows, cols = x.shape
+    if y is None:
+        y = torch.empty(rows, dtype=torch.float32, device=x.device)
+    _check(_lib.pd_reducemean(_dev(x, torch.float32, "x"), _dev(y, torch.float32, "y"), rows, cols, _stream(stream)),
+           "pd_reducemean")
     return y
 
 

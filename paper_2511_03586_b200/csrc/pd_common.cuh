@@ -107,6 +107,7 @@ pd_status launch_layernorm(const float* x, const float* gamma, const float* beta
                            int64_t rows, int64_t cols, float eps, cudaStream_t s);
 pd_status launch_rmsnorm(const float* x, const float* gamma, float* y, int64_t rows, int64_t cols, float eps,
                          cudaStream_t s);
+pd_status launch_reducemean(const float* x, float* y, int64_t rows, int64_t cols, cudaStream_t s);
 pd_status launch_bias_gelu_residual(const float* x, const float* bias, const float* r, float* out,
                                     int64_t rows, int64_t cols, cudaStream_t s);
 

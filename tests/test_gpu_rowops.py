@@ -161,3 +161,30 @@ def test_rowop_errors(api):
         api.pd_softmax(x.double())
     with pytest.raises(TypeError):
         api.pd_softmax(x.cpu())
+
+
+# --------------------------------------------------------------- reducemean
+@pytest.mark.parametrize("shape", [(4096, 4096), (1, 1), (3, 5), (37, 1024), (1000, 512), (129, 1028), (64, 20000), (5, 70001),
+                                   (2, 1 << 20)])
+def test_reducemean_against_oracle(api, shape):
+    rows, cols = shape
+    x = inputs.rmsnorm_inputs(rows, cols, seed=rows + cols)["x"]          # N(1, 2): the mean does not vanish
+    y = Guarded((rows,), torch.float32)
+    api.pd_reducemean(dev_f32(x), y.t)
+    torch.cuda.synchronize()
+    y.check()
+    assert max_rel_floored(host(y.t), oracle.reducemean(x)) < 1e-5
+
+
+def test_reducemean_unaligned_rows_and_exact_integers(api):
+    # a view that starts 4 bytes into an allocation: the scalar path; integer data sums exactly and 1 / 2048 is exact
+    rng = np.random.default_rng(8)
+    x = rng.integers(-1000, 1001, size=(40, 2048)).astype(np.float32)
+    buf = torch.empty(40 * 2048 + 1, dtype=torch.float32, device="cuda")
+    xv = buf[1:].view(40, 2048)
+    xv.copy_(torch.from_numpy(x))
+    y = torch.empty(40, dtype=torch.float32, device="cuda")
+    assert api._lib.pd_reducemean(xv.data_ptr(), y.data_ptr(), 40, 2048, None) == 0
+    ref = oracle.reducemean(x)
+    assert max_rel_floored(host(y), ref) < 1e-6
+    assert np.array_equal(host(api.pd_reducemean(dev_f32(x))), (x.astype(np.float64).sum(axis=1) / 2048).astype(np.float32).astype(np.float64))

@@ -229,6 +229,28 @@ def test_bias_broadcast_residual_and_permutation():
 
 
 # ------------------------------------------------- library cross-check (torch f64)
+# --------------------------------------------------------------- reducemean
+def test_reducemean_closed_forms_and_invariants():
+    # ramp 1..n has mean (n + 1) / 2; a constant row has its constant; integers sum exactly
+    for n in (1, 2, 7, 512, 4096):
+        x = np.arange(1, n + 1, dtype=np.float64).reshape(1, n)
+        np.testing.assert_allclose(oracle.reducemean(x), [(n + 1) / 2], rtol=1e-14)
+    assert np.array_equal(oracle.reducemean(np.full((3, 8), 2.5)), np.full(3, 2.5))
+    rng = np.random.default_rng(51)
+    x = rng.normal(1, 2, size=(6, 333))
+    m = oracle.reducemean(x)
+    assert m.shape == (6,)
+    # rows are independent, the mean is linear, invariant under permutation of a row, shifts with the row
+    np.testing.assert_allclose(oracle.reducemean(3 * x + 1), 3 * m + 1, rtol=1e-13)
+    np.testing.assert_allclose(oracle.reducemean(x[:, rng.permutation(333)]), m, rtol=1e-13)
+    assert np.array_equal(oracle.reducemean(x[2:3]), m[2:3])
+    np.testing.assert_allclose(m, [math.fsum(row) / 333 for row in x], rtol=1e-14)
+    # it is the first statistic of layernorm: subtracting it centres the row the way layernorm does
+    y = oracle.layernorm(x, np.ones(333), np.zeros(333), 0.0)
+    c = x - m[:, None]
+    np.testing.assert_allclose(y, c / np.sqrt((c * c).mean(axis=1, keepdims=True)), rtol=1e-11, atol=1e-13)
+
+
 # ------------------------------------------------------------ relu, swiglu
 def test_relu_epilogue_special_cases():
     x = np.array([[-2.0, -0.0, 0.0, 3.5], [1e-300, -1e-300, 7.0, -7.0]])
