@@ -76,6 +76,66 @@ layernorm_rows_in_registers(const float* __restrict__ x, const float* __restrict
   }
 }
 
+// Rows of 32768 < cols <= 262144: one cluster of up to 8 CTAs per row, the columns dealt evenly, each CTA keeping
+// its share (at most 32 per thread) in registers; 512-thread CTAs, two per SM, up to 131072 columns; the three sums are combined over the cluster through distributed shared memory.
+template <int THREADS, typename OutT>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS)
+layernorm_rows_cluster(const float* __restrict__ x, const float* __restrict__ gamma, const float* __restrict__ beta,
+                       OutT* __restrict__ y, int64_t rows, int cols, float eps) {
+  constexpr int VPT = 8, NWARPS = THREADS / 32;
+  __shared__ float scratch[3][NWARPS];
+  __shared__ float xchg[8];
+  __shared__ __align__(8) float xchg2[16];
+  const int cols4 = cols >> 2;
+  const float inv_cols = 1.0f / (float)cols;
+  const float4* g4 = reinterpret_cast<const float4*>(gamma);
+  const float4* b4 = reinterpret_cast<const float4*>(beta);
+  const int64_t row = blockIdx.x / cluster_size();
+  const int chunk4 = (cols4 + (int)cluster_size() - 1) / (int)cluster_size();  // float4 per CTA, at most VPT * THREADS
+  const int base = (int)cluster_rank() * chunk4;
+  const int end = min(base + chunk4, cols4);
+  griddep_wait();
+  griddep_launch_dependents();
+  const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
+  float4 v[VPT];
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int c = base + threadIdx.x + i * THREADS;
+    v[i] = (c < end) ? ld_stream(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+  const float mu0 = cluster_allreduce<false>(block_reduce<NWARPS, false>(s, scratch, 0), xchg) * inv_cols;
+  // centre on the first estimate and refine it with the mean of the residuals, as in the single-CTA kernel
+  float d1 = 0.f, d2 = 0.f;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int c = base + threadIdx.x + i * THREADS;
+    if (c < end) {
+      v[i].x -= mu0; v[i].y -= mu0; v[i].z -= mu0; v[i].w -= mu0;
+      d1 += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+      d2 += (v[i].x * v[i].x + v[i].y * v[i].y) + (v[i].z * v[i].z + v[i].w * v[i].w);
+    }
+  }
+  d1 = block_reduce<NWARPS, false>(d1, scratch, 1);
+  d2 = block_reduce<NWARPS, false>(d2, scratch, 2);
+  const float2 dd = cluster_allreduce_sum2(d1, d2, xchg2);
+  const float delta = dd.x * inv_cols;
+  const float var = fmaxf(dd.y * inv_cols - delta * delta, 0.f);
+  const float rstd = rsqrtf(var + eps);
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int c = base + threadIdx.x + i * THREADS;
+    if (c < end) {
+      const float4 g = __ldg(g4 + c), b = __ldg(b4 + c);
+      store_out4(y, row * cols4 + c,
+                 make_float4((v[i].x - delta) * rstd * g.x + b.x, (v[i].y - delta) * rstd * g.y + b.y,
+                             (v[i].z - delta) * rstd * g.z + b.z, (v[i].w - delta) * rstd * g.w + b.w));
+    }
+  }
+}
+
 // (count, mean, M2) partial statistics and their pairwise merge.
 struct Moments {
   float n, mean, m2;
@@ -204,13 +264,23 @@ pd_status dispatch(const float* x, const float* g, const float* b, OutT* y, int6
     else if (c <= 256) launch_warp_rows<2>(x, g, b, y, rows, c, eps, s);
     else if (c <= 512) launch_warp_rows<4>(x, g, b, y, rows, c, eps, s);
     else launch_warp_rows<8>(x, g, b, y, rows, c, eps, s);
-  } else if (vec_ok && cols <= 32768) {
+  } else if (vec_ok && cols <= 16384) {  // beyond: two 512-thread CTAs per SM beat one of 1024
     const int c = (int)cols;
     if (c <= 2048) launch_cta_rows<64>(x, g, b, y, rows, c, eps, s);
     else if (c <= 4096) launch_cta_rows<128>(x, g, b, y, rows, c, eps, s);
     else if (c <= 8192) launch_cta_rows<256>(x, g, b, y, rows, c, eps, s);
     else if (c <= 16384) launch_cta_rows<512>(x, g, b, y, rows, c, eps, s);
     else launch_cta_rows<1024>(x, g, b, y, rows, c, eps, s);
+  } else if (vec_ok && cols <= 262144 && rows * 8 <= 0x7fffffff) {
+    if (cols <= 131072) {
+      const unsigned cl = (unsigned)((cols + 16383) / 16384);
+      launch_pdl_cluster(layernorm_rows_cluster<512, OutT>, dim3((unsigned)rows * cl), dim3(512), cl, 0, s, x, g, b, y, rows,
+                         (int)cols, eps);
+    } else {
+      const unsigned cl = (unsigned)((cols + 32767) / 32768);
+      launch_pdl_cluster(layernorm_rows_cluster<1024, OutT>, dim3((unsigned)rows * cl), dim3(1024), cl, 0, s, x, g, b, y, rows,
+                         (int)cols, eps);
+    }
   } else if (vec_ok && x != reinterpret_cast<const float*>(y)) {
     const int grid = (int)(rows < (int64_t)sm_count() * 4 ? rows : (int64_t)sm_count() * 4);
     layernorm_rows_streaming<OutT><<<grid, 512, 0, s>>>(x, g, b, y, rows, cols, eps);

@@ -43,6 +43,27 @@ inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// The same with the CTAs grouped into thread-block clusters of `cluster` along x (grid.x a multiple of it).
+template <typename... KArgs, typename... Args>
+inline void launch_pdl_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, unsigned cluster, size_t smem,
+                               cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = cluster;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ---- device side ---------------------------------------------------------
@@ -76,6 +97,57 @@ __device__ __forceinline__ float block_reduce(float v, float (*scratch)[NWARPS],
   float r = scratch[slot][0];
 #pragma unroll
   for (int w = 1; w < NWARPS; ++w) r = IS_MAX ? fmaxf(r, scratch[slot][w]) : r + scratch[slot][w];
+  return r;
+}
+
+// ---- rows shared by the CTAs of a thread-block cluster ----------------------------
+// Rows too long for one CTA's registers are held by a cluster: CTA r keeps columns [r * chunk, (r + 1) * chunk)
+// and the row statistics are combined through distributed shared memory.
+__device__ __forceinline__ unsigned cluster_rank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ unsigned cluster_size() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+  return r;
+}
+// All-reduce over the cluster of one value per CTA (`v`, identical in all threads of the CTA): thread k writes it
+// into slot [own rank] of CTA k's exchange array, a cluster barrier (release / acquire) publishes the writes,
+// and everyone combines the slots in rank order.  `xchg`: 8 floats of shared memory used by no other reduction.
+template <bool IS_MAX>
+__device__ __forceinline__ float cluster_allreduce(float v, float* xchg) {
+  const unsigned n = cluster_size(), rank = cluster_rank();
+  if (threadIdx.x < n) {
+    const unsigned local = static_cast<unsigned>(__cvta_generic_to_shared(xchg + rank));
+    unsigned remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(threadIdx.x));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+  }
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  float r = xchg[0];
+  for (unsigned k = 1; k < n; ++k) r = IS_MAX ? fmaxf(r, xchg[k]) : r + xchg[k];
+  return r;
+}
+
+// Two sums at once (one barrier): `xchg` holds 16 floats.
+__device__ __forceinline__ float2 cluster_allreduce_sum2(float a, float b, float* xchg) {
+  const unsigned n = cluster_size(), rank = cluster_rank();
+  if (threadIdx.x < n) {
+    const unsigned local = static_cast<unsigned>(__cvta_generic_to_shared(xchg + 2 * rank));
+    unsigned remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(threadIdx.x));
+    asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(remote), "f"(a), "f"(b) : "memory");
+  }
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  float2 r = make_float2(xchg[0], xchg[1]);
+  for (unsigned k = 1; k < n; ++k) {
+    r.x += xchg[2 * k];
+    r.y += xchg[2 * k + 1];
+  }
   return r;
 }
 

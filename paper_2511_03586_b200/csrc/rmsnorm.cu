@@ -6,7 +6,7 @@
 // HBM-bound, 8 bytes per element: the row is read once into registers with
 // 128-bit streaming loads, the sum of squares is reduced with warp shuffles (and
 // through shared memory when several warps share a row), and the row is written
-// once.  Same three paths as the LayerNorm kernel.
+// once.  Same paths as the LayerNorm kernel: a warp, a CTA or a cluster of CTAs per row, by row length.
 #include "pd_common.cuh"
 
 namespace pd {
@@ -47,6 +47,46 @@ rmsnorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__
         store_out4(y, row * cols4 + c,
                    make_float4(v[i].x * rstd * g.x, v[i].y * rstd * g.y, v[i].z * rstd * g.z, v[i].w * rstd * g.w));
       }
+    }
+  }
+}
+
+// Rows of 32768 < cols <= 262144: one cluster of up to 8 CTAs per row, the columns dealt evenly, each CTA keeping
+// its share (at most 32 per thread) in registers; 512-thread CTAs, two per SM, up to 131072 columns; the sum of squares is combined over the cluster through distributed shared memory.
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS)
+rmsnorm_rows_cluster(const float* __restrict__ x, const float* __restrict__ gamma, float* __restrict__ y, int64_t rows,
+                     int cols, float eps) {
+  constexpr int VPT = 8, NWARPS = THREADS / 32;
+  __shared__ float scratch[2][NWARPS];
+  __shared__ float xchg[8];
+  const int cols4 = cols >> 2;
+  const float4* g4 = reinterpret_cast<const float4*>(gamma);
+  const int64_t row = blockIdx.x / cluster_size();
+  const int chunk4 = (cols4 + (int)cluster_size() - 1) / (int)cluster_size();  // float4 per CTA, at most VPT * THREADS
+  const int base = (int)cluster_rank() * chunk4;
+  const int end = min(base + chunk4, cols4);
+  griddep_wait();
+  griddep_launch_dependents();
+  const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
+  float4 v[VPT];
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int c = base + threadIdx.x + i * THREADS;
+    v[i] = (c < end) ? ld_stream(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) q += (v[i].x * v[i].x + v[i].y * v[i].y) + (v[i].z * v[i].z + v[i].w * v[i].w);
+  q = cluster_allreduce<false>(block_reduce<NWARPS, false>(q, scratch, 0), xchg);
+  const float rstd = rsqrtf(q / (float)cols + eps);
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int c = base + threadIdx.x + i * THREADS;
+    if (c < end) {
+      const float4 g = __ldg(g4 + c);
+      store_out4(y, row * cols4 + c,
+                 make_float4(v[i].x * rstd * g.x, v[i].y * rstd * g.y, v[i].z * rstd * g.z, v[i].w * rstd * g.w));
     }
   }
 }
@@ -96,6 +136,14 @@ pd_status launch_rmsnorm(const float* x, const float* g, float* y, int64_t rows,
     else if (c <= 8192) launch_cta_rows<256>(x, g, y, rows, c, eps, s);
     else if (c <= 16384) launch_cta_rows<512>(x, g, y, rows, c, eps, s);
     else launch_cta_rows<1024>(x, g, y, rows, c, eps, s);
+  } else if (vec_ok && cols <= 262144 && rows * 8 <= 0x7fffffff) {
+    if (cols <= 131072) {
+      const unsigned cl = (unsigned)((cols + 16383) / 16384);
+      launch_pdl_cluster(rmsnorm_rows_cluster<512>, dim3((unsigned)rows * cl), dim3(512), cl, 0, s, x, g, y, rows, c, eps);
+    } else {
+      const unsigned cl = (unsigned)((cols + 32767) / 32768);
+      launch_pdl_cluster(rmsnorm_rows_cluster<1024>, dim3((unsigned)rows * cl), dim3(1024), cl, 0, s, x, g, y, rows, c, eps);
+    }
   } else {
     const int grid = (int)(rows < (int64_t)sm_count() * 16 ? rows : (int64_t)sm_count() * 16);
     rmsnorm_rows_generic<<<grid, 256, 0, s>>>(x, g, y, rows, cols, eps);

@@ -7,6 +7,8 @@
 // warp shuffles, and written once.
 //   * cols <= 1024            : one warp per row (up to 8 float4 per lane)
 //   * cols <= 32768           : one CTA of 64 to 1024 threads per row (8 float4 per thread)
+//   * cols <= 262144          : one cluster of 2, 4 or 8 such CTAs per row (statistics combined through
+//                               distributed shared memory)
 //   * longer, 16-byte aligned : one CTA per row, online (max, sum) pass from HBM, normalising pass from L2
 //   * anything else / ragged  : one CTA per row, three scalar passes from global/L2
 #include "pd_common.cuh"
@@ -60,6 +62,52 @@ softmax_rows_in_registers(const float* __restrict__ x, OutT* __restrict__ y, int
         store_out4(y, row * cols4 + c, make_float4(v[i].x * inv, v[i].y * inv, v[i].z * inv, v[i].w * inv));
     }
     if constexpr (NWARPS > 1) __syncthreads();  // scratch is reused by the next row
+  }
+}
+
+// Rows of 32768 < cols <= 262144: one cluster of up to 8 CTAs per row, the columns dealt evenly, each CTA keeping
+// its share (at most 32 per thread) in registers; 512-thread CTAs, two per SM, up to 131072 columns; maximum and sum are combined over the cluster through distributed shared memory,
+// so the row is still read once and written once.
+template <int THREADS, typename OutT>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS)
+softmax_rows_cluster(const float* __restrict__ x, OutT* __restrict__ y, int64_t rows, int cols) {
+  constexpr int VPT = 8, NWARPS = THREADS / 32;
+  __shared__ float scratch[2][NWARPS];
+  __shared__ float xchg[2][8];
+  const int cols4 = cols >> 2;
+  const int64_t row = blockIdx.x / cluster_size();
+  const int chunk4 = (cols4 + (int)cluster_size() - 1) / (int)cluster_size();  // float4 per CTA, at most VPT * THREADS
+  const int base = (int)cluster_rank() * chunk4;
+  const int end = min(base + chunk4, cols4);
+  griddep_wait();
+  griddep_launch_dependents();
+  const float4* xr = reinterpret_cast<const float4*>(x + row * cols);
+  float4 v[VPT];
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int c = base + threadIdx.x + i * THREADS;
+    v[i] = (c < end) ? ld_stream(xr + c) : make_float4(kNegInf, kNegInf, kNegInf, kNegInf);
+  }
+  float m = kNegInf;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) m = fmaxf(m, fmaxf(fmaxf(v[i].x, v[i].y), fmaxf(v[i].z, v[i].w)));
+  m = cluster_allreduce<true>(block_reduce<NWARPS, true>(m, scratch, 0), xchg[0]);
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    v[i].x = expf(v[i].x - m);
+    v[i].y = expf(v[i].y - m);
+    v[i].z = expf(v[i].z - m);
+    v[i].w = expf(v[i].w - m);
+    s += (v[i].x + v[i].y) + (v[i].z + v[i].w);
+  }
+  s = cluster_allreduce<false>(block_reduce<NWARPS, false>(s, scratch, 1), xchg[1]);
+  const float inv = 1.0f / s;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int c = base + threadIdx.x + i * THREADS;
+    if (c < end)
+      store_out4(y, row * cols4 + c, make_float4(v[i].x * inv, v[i].y * inv, v[i].z * inv, v[i].w * inv));
   }
 }
 
@@ -144,13 +192,21 @@ pd_status dispatch(const float* x, OutT* y, int64_t rows, int64_t cols, cudaStre
     else if (c <= 256) launch_warp_rows<2>(x, y, rows, c, s);
     else if (c <= 512) launch_warp_rows<4>(x, y, rows, c, s);
     else launch_warp_rows<8>(x, y, rows, c, s);
-  } else if (vec_ok && cols <= 32768) {
+  } else if (vec_ok && cols <= 16384) {  // beyond: two 512-thread CTAs per SM beat one of 1024
     const int c = (int)cols;
     if (c <= 2048) launch_cta_rows<64>(x, y, rows, c, s);
     else if (c <= 4096) launch_cta_rows<128>(x, y, rows, c, s);
     else if (c <= 8192) launch_cta_rows<256>(x, y, rows, c, s);
     else if (c <= 16384) launch_cta_rows<512>(x, y, rows, c, s);
     else launch_cta_rows<1024>(x, y, rows, c, s);
+  } else if (vec_ok && cols <= 262144 && rows * 8 <= 0x7fffffff) {
+    if (cols <= 131072) {
+      const unsigned cl = (unsigned)((cols + 16383) / 16384);
+      launch_pdl_cluster(softmax_rows_cluster<512, OutT>, dim3((unsigned)rows * cl), dim3(512), cl, 0, s, x, y, rows, (int)cols);
+    } else {
+      const unsigned cl = (unsigned)((cols + 32767) / 32768);
+      launch_pdl_cluster(softmax_rows_cluster<1024, OutT>, dim3((unsigned)rows * cl), dim3(1024), cl, 0, s, x, y, rows, (int)cols);
+    }
   } else if (vec_ok && x != reinterpret_cast<const float*>(y)) {
     const int grid = (int)(rows < (int64_t)sm_count() * 4 ? rows : (int64_t)sm_count() * 4);
     softmax_rows_streaming<OutT><<<grid, 512, 0, s>>>(x, y, rows, cols);
