@@ -264,7 +264,7 @@ pd_status dispatch(const float* x, const float* g, const float* b, OutT* y, int6
     else if (c <= 256) launch_warp_rows<2>(x, g, b, y, rows, c, eps, s);
     else if (c <= 512) launch_warp_rows<4>(x, g, b, y, rows, c, eps, s);
     else launch_warp_rows<8>(x, g, b, y, rows, c, eps, s);
-  } else if (vec_ok && cols <= 16384) {  // beyond: two 512-thread CTAs per SM beat one of 1024
+  } else if (vec_ok && cols <= 28672) {  // beyond (measured): a cluster of 512-thread CTAs, two per SM, is faster
     const int c = (int)cols;
     if (c <= 2048) launch_cta_rows<64>(x, g, b, y, rows, c, eps, s);
     else if (c <= 4096) launch_cta_rows<128>(x, g, b, y, rows, c, eps, s);
