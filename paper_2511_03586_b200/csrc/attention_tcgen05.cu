@@ -142,7 +142,7 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
       mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1);
       mbar_init(o_full(s), 1); mbar_init(o_empty(s), kSlotThreads);
       for (int b = 0; b < 2; ++b) {
-        mbar_init(s_full(s, b), 1); mbar_init(s_empty(s, b), kSlotThreads);
+        mbar_init(s_full(s, b), 1); mbar_init(s_empty(s, b), 1);
         mbar_init(p_full(s, b), kSlotThreads); mbar_init(p_empty(s, b), 1);
       }
     }
@@ -249,7 +249,6 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
     if (lane < kSlots) {
       const int s = lane;
       constexpr uint32_t idesc_o = make_idesc_bf16(kBlockQ, kD, false, true);  // V is MN-major
-      const uint64_t p_desc = make_smem_desc(sP + 2 * s * kSmemP, 0, 1024);
       const uint64_t v_desc = make_smem_desc(sV, 0, 1024);
       const uint32_t d_tmem = tmem_base + kTmemO + s * kD;
       uint32_t t = 0, n_us = 0, n_unit = 0;
@@ -265,12 +264,14 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
             const uint32_t buf = t & 1u;
             if (!mbar_wait(p_full(s, buf), (t >> 1) & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
             tcgen05_fence_after_sync();
-            const uint64_t pg = p_desc + (uint64_t)(buf * (kSmemP >> 4));
+            // P_g sits in tensor memory, over the first 32 columns of the score buffer it was computed from
+            const uint32_t pg = tmem_base + kTmemS + s * 128 + buf * kBlockK;
             const uint64_t vg = v_desc + (uint64_t)(g * ((kBlockK * 128) >> 4));
 #pragma unroll
             for (int ks = 0; ks < kBlockK / 16; ++ks)
-              mma_bf16_ss(d_tmem, pg + 2 * ks, vg + ks * ((16 * 128) >> 4), idesc_o, (g | ks) != 0 ? 1u : 0u);
+              mma_bf16_ts(d_tmem, pg + 8 * ks, vg + ks * ((16 * 128) >> 4), idesc_o, (g | ks) != 0 ? 1u : 0u);
             mma_commit(p_empty(s, buf));
+            mma_commit(s_empty(s, buf));  // the score buffer (and P inside it) may be overwritten
           }
           if (!ok) break;
           mma_commit(o_full(s));
@@ -303,7 +304,6 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         const int buf = t & 1u;
         const uint32_t use_ph = (t >> 1) & 1u;
         const uint32_t t_s = t_lane + kTmemS + slot * 128 + buf * kBlockK;
-        const uint32_t p_row = sP + (2 * slot + buf) * kSmemP + (uint32_t)row * 128u;
         const int key0 = g * kBlockK;
         if (!mbar_wait(s_full(slot, buf), use_ph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
         tcgen05_fence_after_sync();
@@ -329,10 +329,11 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
           __syncwarp();
           store_pending = false;
         }
-        // P_{g-2} V_{g-2} read the tile rewritten below: it must have completed
-        if (!mbar_wait(p_empty(slot, buf), use_ph ^ 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+        // (P_g goes over the score buffer it came from; the product that read the buffer's previous contents
+        // completed before the scores were written)
         // exponentials of the block against reference `ref`: writes P and returns the row's partial sum
         // (two fp32 values per instruction where the operation exists in packed form)
+        uint32_t pk[kBlockK / 2];  // the block's probabilities, two bf16 per register
         auto exp_block = [&](float ref) {
           uint64_t part2[2] = {0, 0};
           float part = 0.f;
@@ -345,7 +346,6 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
             if (cc + 1 < kBlockK / 32) tmem_ld_32x32b_x32(t_s + (cc + 1) * 32, r[(cc & 1) ^ 1]);
             const uint32_t(&rr)[32] = r[cc & 1];
             const int c0 = key0 + cc * 32;
-            uint32_t pk[16];
             if (c0 + 32 <= p.seq) {
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
@@ -370,7 +370,7 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
                   e1 = ex2_approx(a1);
                 }
                 part2[(i >> 1) & 1] = add_f32x2(part2[(i >> 1) & 1], pack_f32x2(e0, e1));
-                pk[i / 2] = pack_bf16x2(e0, e1);
+                pk[cc * 16 + i / 2] = pack_bf16x2(e0, e1);
               }
             } else {
 #pragma unroll
@@ -380,14 +380,9 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
                 const float e0 = c0 + i < p.seq ? ex2_approx(a0) : 0.f;
                 const float e1 = c0 + i + 1 < p.seq ? ex2_approx(a1) : 0.f;
                 part += e0 + e1;
-                pk[i / 2] = pack_bf16x2(e0, e1);
+                pk[cc * 16 + i / 2] = pack_bf16x2(e0, e1);
               }
             }
-            // keys 32*cc .. 32*cc+31 of the block: 16-byte units 4*cc .. 4*cc+3 of the row
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-              st_shared_v4(p_row + (((uint32_t)(4 * cc + u) ^ sw) << 4),
-                           make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]));
           }
           float s0, s1;
           unpack_f32x2(add_f32x2(part2[0], part2[1]), s0, s1);
@@ -436,10 +431,11 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
           part = exp_block(mk);
         }
         l += part;
-        fence_proxy_async_smem();
+        // P_g replaces the scores it was computed from (keys 2j, 2j + 1 in column j: the A operand of P V)
+        tmem_st_32x32b_x32(t_s, pk);
+        tmem_st_wait();
         tcgen05_fence_before_sync();
         mbar_arrive(p_full(slot, buf));
-        mbar_arrive(s_empty(slot, buf));
       }
       if (!ok) break;
       // ---- output: O / l -> bf16 -> the slot's first probability tile (free by now: every P V product
