@@ -5,43 +5,46 @@
 // on the packed projection qkv[tokens, 3*hidden] = [Q | K | V].  Scores and
 // probabilities never leave the SM.
 //
-// One persistent CTA of 352 threads per SM walks over work units of (batch,
+// One persistent CTA of 416 threads per SM walks over work units of (batch,
 // head, pair of 128-query blocks).  K and V of the head (up to 512 x 64 each)
-// are resident in shared memory for the unit; the two query blocks ("slots")
-// are in flight at the same time, and each slot works through the keys in
-// blocks of 64 with two score buffers in tensor memory and two probability
-// tiles in shared memory, so that the tensor core, the exponential unit and the
-// barrier round trips overlap.  The stream of blocks runs on across unit
-// boundaries: the first score product of the next unit is issued while the
-// last blocks of the current one are still being exponentiated.
+// sit in shared memory in four chunks of 128 keys, each with its own full and
+// empty barrier, so that the next unit's chunks stream in while the current
+// unit is still working on the later ones; the query tiles are double
+// buffered for the same reason.  The two query blocks ("slots") are in flight
+// at the same time, and each slot works through the keys in blocks of 64 with
+// two score buffers, two probability buffers and one output accumulator in
+// tensor memory (all 512 columns), so that the tensor core, the exponential
+// unit and the barrier round trips overlap, also across unit boundaries.
 //
-//   warp 8, one lane : TMA producer (K, V once per unit; Q once per slot).
-//   warp 9, lanes 0-1: score issuers, one thread per slot: for block g of
+//   warp 8, one lane : TMA producer (per unit: Q of each slot, then the K and V
+//                      chunks in the order the previous unit releases them).
+//   warps 9, 11      : score issuers, one thread per slot, each in a warp of
+//                      its own (see kProducerWarp below): for block g of
 //                      64 keys S = Q K_g^T (128 x 64 x 64) into one of the slot's
-//                      two score buffers, as soon as that buffer is free; they
-//                      run ahead of the softmax by up to two blocks, also across
-//                      unit boundaries.
-//   warp 10, lanes 0-1: output issuers, one thread per slot: when the
+//                      two score buffers, as soon as the softmax warps have
+//                      read that buffer's previous contents.
+//   warps 10, 12     : output issuers, one thread per slot: when the
 //                      slot's softmax warps have published P_g,
 //                      O += P_g V_g (128 x 64 x 64) into the slot's 64 output
-//                      columns.  (A single issuing thread for all four streams
+//                      columns, P_g read from tensor memory as the A operand.
+//                      (A single issuing thread for all four streams
 //                      was the bottleneck: the per-product bookkeeping of one
 //                      thread cost more than the products themselves.)
 //   warps 0-3, 4-7   : softmax of slot 0 / slot 1, one thread per query row.
 //                      The row keeps a reference exponent m (the maximum of its
 //                      first block).  For each block it forms
 //                      p = 2^(s * log2(e) / 8 - m) from the scores in tensor
-//                      memory, adds them to the fp32 row sum l and writes P as
-//                      bf16 into the swizzled shared-memory tile the MMA reads
-//                      as its A operand.  While doing so it tracks the largest
-//                      exponent of the block; only if that exceeds 16 (p would
-//                      still be far from overflow) is m raised, O and l rescaled
+//                      memory, adds them to the fp32 row sum l, releases the
+//                      score buffer and writes P as bf16 into the probability
+//                      buffer.  The block's sum shows whether any exponent
+//                      exceeded 16 (p would
+//                      still be far from overflow); only then is m raised, O and l rescaled
 //                      by 2^(m_old - m_new) through a tensor-memory load / store
 //                      round trip, and the block redone.  O / l is therefore the
 //                      exact softmax for any finite input, and on ordinary
 //                      inputs every score is read once.  Finally the thread
 //                      reads its O row, divides by l and stages 64 bf16 values
-//                      in the (by then idle) probability tile, from where each
+//                      in shared memory, from where each
 //                      warp's 32 rows go to Ctx with one TMA store.
 // Keys beyond the sequence length are zero-filled by TMA and masked out; query
 // rows beyond it are computed and discarded.
@@ -60,19 +63,28 @@ constexpr int kBlockQ = 128;      // queries per slot = TMEM lanes
 constexpr int kBlockK = 64;       // keys per score block
 constexpr int kMaxKeys = 512;
 constexpr int kSlots = 2;         // query blocks in flight
-constexpr int kThreads = 352;
+constexpr int kThreads = 416;
 constexpr int kSlotThreads = 128;
-constexpr int kProducerWarp = 8, kScoreWarp = 9, kOutputWarp = 10, kAllocWarp = 9;
+// warps 0-7 softmax; then one warp per single-thread role.  Every tcgen05.mma / tcgen05.commit issuing thread has a
+// warp of its own: two lanes of one warp that reach the same tcgen05 instruction together, with different
+// operands, do not get two independent operations (attention with peaked rows came out wrong that way whenever
+// the two slots drifted apart).
+constexpr int kProducerWarp = 8, kScoreWarp0 = 9, kOutputWarp0 = 10, kScoreWarp1 = 11, kOutputWarp1 = 12;
+constexpr int kAllocWarp = kScoreWarp0;
 
 constexpr int kSmemK = kMaxKeys * kD * 2;        // 64 KiB
 constexpr int kSmemV = kMaxKeys * kD * 2;        // 64 KiB
-constexpr int kSmemQ = kBlockQ * kD * 2;         // 16 KiB per slot
-constexpr int kSmemP = kBlockQ * kBlockK * 2;    // 16 KiB per probability tile, two per slot
+constexpr int kSmemQ = kBlockQ * kD * 2;         // 16 KiB per query tile, two per slot
+constexpr int kSmemO = kBlockQ * kD * 2;         // 16 KiB of output staging per slot
+constexpr int kChunkKeys = 128;                  // K and V arrive, and are released, in chunks of 128 keys
+constexpr int kChunks = kMaxKeys / kChunkKeys;
+constexpr int kSmemChunk = kChunkKeys * kD * 2;  // 16 KiB
 constexpr int kSmemCtrl = 1024;
-constexpr int kSmemBytes = kSmemK + kSmemV + kSlots * (kSmemQ + 2 * kSmemP) + kSmemCtrl + 1024 /*alignment slack*/;
+constexpr int kSmemBytes = kSmemK + kSmemV + kSlots * (2 * kSmemQ + kSmemO) + kSmemCtrl + 1024 /*alignment slack*/;
 
-// tensor-memory columns: score buffer b of slot s at 128*s + 64*b, output accumulator of slot s at 256 + 64*s
-constexpr uint32_t kTmemS = 0, kTmemO = 256, kTmemCols = 512;
+// tensor-memory columns: score buffer b of slot s at 128*s + 64*b, output accumulator of slot s at 256 + 64*s,
+// probability buffer b of slot s (64 bf16 per row in 32 columns) at 384 + 64*s + 32*b
+constexpr uint32_t kTmemS = 0, kTmemO = 256, kTmemP = 384, kTmemCols = 512;
 
 constexpr float kScale = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
 constexpr float kRescaleThreshold = 16.0f;               // largest exponent of 2 tolerated before m is raised
@@ -116,19 +128,22 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t sK = smem_base, sV = sK + kSmemK, sQ = sV + kSmemV, sP = sQ + kSlots * kSmemQ;
-  const uint32_t bar_base = sP + kSlots * 2 * kSmemP;
-  // barriers (8 bytes each); [s] = slot, [s][b] = slot and buffer
-  const uint32_t k_full = bar_base + 0, v_full = bar_base + 8, k_empty = bar_base + 16, v_empty = bar_base + 24;
-  auto q_full = [&](int s) { return bar_base + 40u + 8u * s; };
-  auto q_empty = [&](int s) { return bar_base + 56u + 8u * s; };
-  auto o_full = [&](int s) { return bar_base + 72u + 8u * s; };
-  auto o_empty = [&](int s) { return bar_base + 88u + 8u * s; };
-  auto s_full = [&](int s, int b) { return bar_base + 104u + 8u * (2 * s + b); };
-  auto s_empty = [&](int s, int b) { return bar_base + 136u + 8u * (2 * s + b); };
-  auto p_full = [&](int s, int b) { return bar_base + 168u + 8u * (2 * s + b); };
-  auto p_empty = [&](int s, int b) { return bar_base + 200u + 8u * (2 * s + b); };
-  const uint32_t drain_bar = bar_base + 232;  // four of them, one per MMA-issuing warp
+  const uint32_t sK = smem_base, sV = sK + kSmemK, sQ = sV + kSmemV, sO = sQ + kSlots * 2 * kSmemQ;
+  const uint32_t bar_base = sO + kSlots * kSmemO;
+  // barriers (8 bytes each); [c] = chunk of 128 keys, [s] = slot, [s][b] = slot and buffer
+  auto k_full = [&](int c) { return bar_base + 8u * c; };
+  auto k_empty = [&](int c) { return bar_base + 32u + 8u * c; };
+  auto v_full = [&](int c) { return bar_base + 64u + 8u * c; };
+  auto v_empty = [&](int c) { return bar_base + 96u + 8u * c; };
+  auto q_full = [&](int s, int b) { return bar_base + 128u + 8u * (2 * s + b); };
+  auto q_empty = [&](int s, int b) { return bar_base + 160u + 8u * (2 * s + b); };
+  auto o_full = [&](int s) { return bar_base + 192u + 8u * s; };
+  auto o_empty = [&](int s) { return bar_base + 208u + 8u * s; };
+  auto s_full = [&](int s, int b) { return bar_base + 224u + 8u * (2 * s + b); };
+  auto s_empty = [&](int s, int b) { return bar_base + 256u + 8u * (2 * s + b); };
+  auto p_full = [&](int s, int b) { return bar_base + 288u + 8u * (2 * s + b); };
+  auto p_empty = [&](int s, int b) { return bar_base + 320u + 8u * (2 * s + b); };
+  const uint32_t drain_bar = bar_base + 352;  // four of them, one per MMA-issuing thread
   uint8_t* ctrl = smem_gen + (bar_base - smem_base) + 512;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 4);
@@ -136,14 +151,16 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    mbar_init(k_full, 1); mbar_init(v_full, 1); mbar_init(k_empty, kSlots); mbar_init(v_empty, kSlots);
+    for (int c = 0; c < kChunks; ++c) {
+      mbar_init(k_full(c), 1); mbar_init(v_full(c), 1); mbar_init(k_empty(c), kSlots); mbar_init(v_empty(c), kSlots);
+    }
     for (int i = 0; i < 4; ++i) mbar_init(drain_bar + 8u * i, 1);
     for (int s = 0; s < kSlots; ++s) {
-      mbar_init(q_full(s), 1); mbar_init(q_empty(s), 1);
-      mbar_init(o_full(s), 1); mbar_init(o_empty(s), kSlotThreads);
+      mbar_init(o_full(s), 1); mbar_init(o_empty(s), (kSlotThreads / 32));
       for (int b = 0; b < 2; ++b) {
-        mbar_init(s_full(s, b), 1); mbar_init(s_empty(s, b), 1);
-        mbar_init(p_full(s, b), kSlotThreads); mbar_init(p_empty(s, b), 1);
+        mbar_init(q_full(s, b), 1); mbar_init(q_empty(s, b), 1);
+        mbar_init(s_full(s, b), 1); mbar_init(s_empty(s, b), (kSlotThreads / 32));
+        mbar_init(p_full(s, b), (kSlotThreads / 32)); mbar_init(p_empty(s, b), 1);
       }
     }
     *abort_flag = 0;
@@ -172,46 +189,67 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
     nslots = min(kSlots, p.q_blocks - qb0);
   };
   const int G = p.k_blocks;
+  const int NC = (G + 1) >> 1;  // chunks of 128 keys in use; chunk c holds score blocks 2c and 2c + 1
 
   if (warp == kProducerWarp) {
     // ------------------------------------------------------------- TMA producer
+    // Per unit: the two query tiles (into the slot's other buffer, normally free long before), then the chunks
+    // of K and V in the order in which the previous unit releases them.
     if (lane == 0) {
       prefetch_tensormap(&tmap_q); prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v);
-      uint32_t n_unit = 0, n_q0 = 0, n_q1 = 0;
+      uint32_t n_unit = 0, n_q[kSlots] = {0, 0};
+      uint32_t armed_k = 0, armed_v = 0;  // bit c: chunk c of the current unit has been requested
       bool ok = true;
+      auto load_k = [&](int c, int h, int b) {
+        if (c >= NC || !ok) return;
+        if (!mbar_wait(k_empty(c), (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; return; }
+        mbar_arrive_expect_tx(k_full(c), kSmemChunk);
+        tma_load_4d(sK + c * kSmemChunk, &tmap_k, k_full(c), 0, c * kChunkKeys, h, b);
+        armed_k |= 1u << c;
+      };
+      auto load_v = [&](int c, int h, int b) {
+        if (c >= NC || !ok) return;
+        if (!mbar_wait(v_empty(c), (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; return; }
+        mbar_arrive_expect_tx(v_full(c), kSmemChunk);
+        tma_load_4d(sV + c * kSmemChunk, &tmap_v, v_full(c), 0, c * kChunkKeys, h, b);
+        armed_v |= 1u << c;
+      };
       for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x, ++n_unit) {
         int b, h, qb0, nslots;
         unit_coords(unit, b, h, qb0, nslots);
-        if (!mbar_wait(k_empty, (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
-        mbar_arrive_expect_tx(k_full, kSmemK);
-        tma_load_4d(sK, &tmap_k, k_full, 0, 0, h, b);
-        tma_load_4d(sK + kSmemK / 2, &tmap_k, k_full, 0, 256, h, b);
+        armed_k = armed_v = 0;
         for (int s = 0; s < nslots && ok; ++s) {
-          const uint32_t nq = s ? n_q1 : n_q0;
-          if (!mbar_wait(q_empty(s), (nq & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
-          if (s) ++n_q1; else ++n_q0;
-          mbar_arrive_expect_tx(q_full(s), kSmemQ);
-          tma_load_4d(sQ + s * kSmemQ, &tmap_q, q_full(s), 0, (qb0 + s) * kBlockQ, h, b);
+          const uint32_t qb = n_q[s] & 1u; const uint32_t qpar = ((n_q[s] >> 1) & 1u) ^ 1u;
+          if (!mbar_wait(q_empty(s, qb), qpar, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
+          ++n_q[s];
+          mbar_arrive_expect_tx(q_full(s, qb), kSmemQ);
+          tma_load_4d(sQ + (2 * s + qb) * kSmemQ, &tmap_q, q_full(s, qb), 0, (qb0 + s) * kBlockQ, h, b);
         }
-        if (!ok) break;
-        if (!mbar_wait(v_empty, (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
-        mbar_arrive_expect_tx(v_full, kSmemV);
-        tma_load_4d(sV, &tmap_v, v_full, 0, 0, h, b);
-        tma_load_4d(sV + kSmemV / 2, &tmap_v, v_full, 0, 256, h, b);
+        load_k(0, h, b); load_k(1, h, b); load_v(0, h, b); load_k(2, h, b); load_v(1, h, b); load_k(3, h, b);
+        load_v(2, h, b); load_v(3, h, b);
+        if (!ok) break;  // n_unit stays the index of the unit that was cut short
       }
-      if (!ok && n_unit > 0) {
-        // leave no copy in flight: give the barriers armed last a short time to complete
+      if (!ok) {
+        // leave no copy in flight: give the latest request on every barrier a short time to land
         volatile int never = 0;
-        mbar_wait(k_full, (n_unit - 1u) & 1u, &never, nullptr, 0, 20000000ull);
-        mbar_wait(v_full, (n_unit - 1u) & 1u, &never, nullptr, 0, 20000000ull);
+        for (int c = 0; c < NC; ++c) {
+          if ((armed_k >> c) & 1u) mbar_wait(k_full(c), n_unit & 1u, &never, nullptr, 0, 20000000ull);
+          else if (n_unit > 0) mbar_wait(k_full(c), (n_unit - 1u) & 1u, &never, nullptr, 0, 20000000ull);
+          if ((armed_v >> c) & 1u) mbar_wait(v_full(c), n_unit & 1u, &never, nullptr, 0, 20000000ull);
+          else if (n_unit > 0) mbar_wait(v_full(c), (n_unit - 1u) & 1u, &never, nullptr, 0, 20000000ull);
+        }
+        for (int s = 0; s < kSlots; ++s)
+          for (uint32_t back = 1; back <= 2 && back <= n_q[s]; ++back) {
+            const uint32_t i = n_q[s] - back;
+            mbar_wait(q_full(s, i & 1u), (i >> 1) & 1u, &never, nullptr, 0, 20000000ull);
+          }
       }
     }
-  } else if (warp == kScoreWarp) {
-    // ---------------------- score-product issuers: lane 0 for slot 0, lane 1 for slot 1
-    if (lane < kSlots) {
-      const int s = lane;
+  } else if (warp == kScoreWarp0 || warp == kScoreWarp1) {
+    // ---------------------- score-product issuers: one thread per slot, each in its own warp
+    if (lane == 0) {
+      const int s = warp == kScoreWarp0 ? 0 : 1;
       constexpr uint32_t idesc_s = make_idesc_bf16(kBlockQ, kBlockK, false, false);  // Q K^T: both K-major
-      const uint64_t q_desc = make_smem_desc(sQ + s * kSmemQ, 0, 1024);
       const uint64_t k_desc = make_smem_desc(sK, 0, 1024);
       const uint32_t d_tmem = tmem_base + kTmemS + s * 128;
       uint32_t t = 0, n_q = 0, n_unit = 0;
@@ -219,24 +257,33 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
       for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x, ++n_unit) {
         int b, h, qb0, nslots;
         unit_coords(unit, b, h, qb0, nslots);
-        if (!mbar_wait(k_full, n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-        if (s < nslots) {
-          if (!mbar_wait(q_full(s), n_q & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+        const bool active = s < nslots;
+        const uint32_t qb = n_q & 1u; const uint32_t qpar = (n_q >> 1) & 1u;
+        uint64_t q_desc = 0;
+        if (active) {
+          if (!mbar_wait(q_full(s, qb), qpar, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
           ++n_q;
-          for (int g = 0; g < G; ++g, ++t) {
-            const uint32_t buf = t & 1u;
-            if (!mbar_wait(s_empty(s, buf), ((t >> 1) & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-            tcgen05_fence_after_sync();
-            const uint64_t kg = k_desc + (uint64_t)(g * ((kBlockK * 128) >> 4));
-#pragma unroll
-            for (int ks = 0; ks < kD / 16; ++ks)
-              mma_bf16_ss(d_tmem + buf * kBlockK, q_desc + 2 * ks, kg + 2 * ks, idesc_s, ks != 0 ? 1u : 0u);
-            mma_commit(s_full(s, buf));
-          }
-          if (!ok) break;
-          mma_commit(q_empty(s));
+          q_desc = make_smem_desc(sQ + (2 * s + qb) * kSmemQ, 0, 1024);
         }
-        mma_commit(k_empty);  // both score issuers arrive, whether or not their slot is in use
+        for (int c = 0; c < NC && ok; ++c) {
+          if (!mbar_wait(k_full(c), n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+          if (active) {
+            for (int g = 2 * c; g < min(2 * c + 2, G); ++g, ++t) {
+              const uint32_t buf = t & 1u;
+              if (!mbar_wait(s_empty(s, buf), ((t >> 1) & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+              tcgen05_fence_after_sync();
+              const uint64_t kg = k_desc + (uint64_t)(g * ((kBlockK * 128) >> 4));
+#pragma unroll
+              for (int ks = 0; ks < kD / 16; ++ks)
+                mma_bf16_ss(d_tmem + buf * kBlockK, q_desc + 2 * ks, kg + 2 * ks, idesc_s, ks != 0 ? 1u : 0u);
+              mma_commit(s_full(s, buf));
+            }
+            if (!ok) break;
+          }
+          mma_commit(k_empty(c));  // both score issuers arrive, whether or not their slot is in use
+        }
+        if (!ok) break;
+        if (active) mma_commit(q_empty(s, qb));
       }
       if (!ok) {
         mma_commit(drain_bar + 16u + 8u * s);
@@ -244,10 +291,10 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         mbar_wait(drain_bar + 16u + 8u * s, 0, &never, nullptr, 0, 20000000ull);
       }
     }
-  } else if (warp == kOutputWarp) {
-    // ------------------------ P V product issuers: lane 0 for slot 0, lane 1 for slot 1
-    if (lane < kSlots) {
-      const int s = lane;
+  } else if (warp == kOutputWarp0 || warp == kOutputWarp1) {
+    // ------------------------ P V product issuers: one thread per slot, each in its own warp
+    if (lane == 0) {
+      const int s = warp == kOutputWarp0 ? 0 : 1;
       constexpr uint32_t idesc_o = make_idesc_bf16(kBlockQ, kD, false, true);  // V is MN-major
       const uint64_t v_desc = make_smem_desc(sV, 0, 1024);
       const uint32_t d_tmem = tmem_base + kTmemO + s * kD;
@@ -256,28 +303,35 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
       for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x, ++n_unit) {
         int b, h, qb0, nslots;
         unit_coords(unit, b, h, qb0, nslots);
-        if (!mbar_wait(v_full, n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-        if (s < nslots) {
+        const bool active = s < nslots;
+        if (active) {
           // the previous unit's output of this slot must have been read before it is overwritten
           if (!mbar_wait(o_empty(s), (n_us & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-          for (int g = 0; g < G; ++g, ++t) {
-            const uint32_t buf = t & 1u;
-            if (!mbar_wait(p_full(s, buf), (t >> 1) & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
-            tcgen05_fence_after_sync();
-            // P_g sits in tensor memory, over the first 32 columns of the score buffer it was computed from
-            const uint32_t pg = tmem_base + kTmemS + s * 128 + buf * kBlockK;
-            const uint64_t vg = v_desc + (uint64_t)(g * ((kBlockK * 128) >> 4));
+        }
+        for (int c = 0; c < NC && ok; ++c) {
+          if (!mbar_wait(v_full(c), n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+          if (active) {
+            for (int g = 2 * c; g < min(2 * c + 2, G); ++g, ++t) {
+              const uint32_t buf = t & 1u;
+              if (!mbar_wait(p_full(s, buf), (t >> 1) & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+              tcgen05_fence_after_sync();
+              // P_g is the A operand straight from tensor memory: keys 2j, 2j + 1 of the block in column j
+              const uint32_t pg = tmem_base + kTmemP + s * 64 + buf * 32;
+              const uint64_t vg = v_desc + (uint64_t)(g * ((kBlockK * 128) >> 4));
 #pragma unroll
-            for (int ks = 0; ks < kBlockK / 16; ++ks)
-              mma_bf16_ts(d_tmem, pg + 8 * ks, vg + ks * ((16 * 128) >> 4), idesc_o, (g | ks) != 0 ? 1u : 0u);
-            mma_commit(p_empty(s, buf));
-            mma_commit(s_empty(s, buf));  // the score buffer (and P inside it) may be overwritten
+              for (int ks = 0; ks < kBlockK / 16; ++ks)
+                mma_bf16_ts(d_tmem, pg + 8 * ks, vg + ks * ((16 * 128) >> 4), idesc_o, (g | ks) != 0 ? 1u : 0u);
+              mma_commit(p_empty(s, buf));
+            }
+            if (!ok) break;
           }
-          if (!ok) break;
+          mma_commit(v_empty(c));  // both output issuers arrive
+        }
+        if (!ok) break;
+        if (active) {
           mma_commit(o_full(s));
           ++n_us;
         }
-        mma_commit(v_empty);  // both output issuers arrive
       }
       if (!ok) {
         mma_commit(drain_bar + 8u * s);
@@ -294,7 +348,7 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
     const uint32_t sw = (uint32_t)(lane & 7);
     uint32_t t = 0, n_us = 0;  // score blocks and units this slot has processed
     bool ok = true;
-    bool store_pending = false;  // this warp's output store may still be reading probability tile 0
+    bool store_pending = false;  // this warp's output store may still be reading the staging tile
     for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x) {
       int b, h, qb0, nslots;
       unit_coords(unit, b, h, qb0, nslots);
@@ -304,6 +358,7 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         const int buf = t & 1u;
         const uint32_t use_ph = (t >> 1) & 1u;
         const uint32_t t_s = t_lane + kTmemS + slot * 128 + buf * kBlockK;
+        const uint32_t t_p = t_lane + kTmemP + slot * 64 + buf * 32;
         const int key0 = g * kBlockK;
         if (!mbar_wait(s_full(slot, buf), use_ph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
         tcgen05_fence_after_sync();
@@ -324,14 +379,7 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
           }
           mk = bm * kScale;
         }
-        if (store_pending && buf == 0) {
-          if (lane == 0) tma_store_wait_read<0>();
-          __syncwarp();
-          store_pending = false;
-        }
-        // (P_g goes over the score buffer it came from; the product that read the buffer's previous contents
-        // completed before the scores were written)
-        // exponentials of the block against reference `ref`: writes P and returns the row's partial sum
+        // exponentials of the block against reference `ref`: fills pk and returns the row's partial sum
         // (two fp32 values per instruction where the operation exists in packed form)
         uint32_t pk[kBlockK / 2];  // the block's probabilities, two bf16 per register
         auto exp_block = [&](float ref) {
@@ -431,21 +479,33 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
           part = exp_block(mk);
         }
         l += part;
-        // P_g replaces the scores it was computed from (keys 2j, 2j + 1 in column j: the A operand of P V)
-        tmem_st_32x32b_x32(t_s, pk);
+        // the scores have been read for good: the buffer may take the block after next
+        tcgen05_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(s_empty(slot, buf));
+        // P_g (keys 2j, 2j + 1 in column j: the A operand of P V) goes to its own tensor-memory buffer once the
+        // product that read the buffer's previous contents has completed
+        if (!mbar_wait(p_empty(slot, buf), use_ph ^ 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+        tcgen05_fence_after_sync();
+        tmem_st_32x32b_x32(t_p, pk);
         tmem_st_wait();
         tcgen05_fence_before_sync();
-        mbar_arrive(p_full(slot, buf));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(p_full(slot, buf));
       }
       if (!ok) break;
-      // ---- output: O / l -> bf16 -> the slot's first probability tile (free by now: every P V product
-      // of the unit has completed) -> one TMA store of 32 rows x 128 bytes per warp; rows beyond the
-      // sequence are clipped by the tensor map
+      // ---- output: O / l -> bf16 -> the slot's staging tile -> one TMA store of 32 rows x 128 bytes per
+      // warp; rows beyond the sequence are clipped by the tensor map
+      if (store_pending) {
+        if (lane == 0) tma_store_wait_read<0>();
+        __syncwarp();
+        store_pending = false;
+      }
       if (!mbar_wait(o_full(slot), n_us & 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
       ++n_us;
       tcgen05_fence_after_sync();
       const float inv = 1.0f / l;
-      const uint32_t o_row = sP + (2 * slot) * kSmemP + (uint32_t)row * 128u;
+      const uint32_t o_row = sO + slot * kSmemO + (uint32_t)row * 128u;
 #pragma unroll
       for (int c0 = 0; c0 < kD; c0 += 32) {
         uint32_t r[32];
@@ -464,13 +524,14 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
       fence_proxy_async_smem();
       __syncwarp();
       if (lane == 0) {
-        tma_store_4d(&tmap_o, sP + (2 * slot) * kSmemP + (uint32_t)(quarter * 32) * 128u, 0,
+        tma_store_4d(&tmap_o, sO + slot * kSmemO + (uint32_t)(quarter * 32) * 128u, 0,
                      (qb0 + slot) * kBlockQ + quarter * 32, h, b);
         tma_store_commit();
       }
       store_pending = true;
       tcgen05_fence_before_sync();
-      mbar_arrive(o_empty(slot));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(o_empty(slot));
     }
     // shared memory must outlive every store that still reads it
     if (lane == 0) tma_store_wait_all<0>();
@@ -510,8 +571,8 @@ pd_status launch_fused_attention(const __nv_bfloat16* qkv, __nv_bfloat16* ctx, i
   const int64_t hidden = heads * kD;
   CUtensorMap tq, tk, tv;
   if (!make_head_map(&tq, qkv, seq, heads, batch, hidden, kBlockQ) ||
-      !make_head_map(&tk, qkv + hidden, seq, heads, batch, hidden, 256) ||
-      !make_head_map(&tv, qkv + 2 * hidden, seq, heads, batch, hidden, 256))
+      !make_head_map(&tk, qkv + hidden, seq, heads, batch, hidden, kChunkKeys) ||
+      !make_head_map(&tv, qkv + 2 * hidden, seq, heads, batch, hidden, kChunkKeys))
     return PD_ERR_UNSUPPORTED;
   // Ctx[batch*seq, hidden] seen as {64, seq, heads, batch}; written in boxes of 32 rows x 64 columns
   CUtensorMap to;

@@ -87,7 +87,9 @@ def test_attention_peaked_rows_and_errors(api):
         qkv[:, :h2 * 64] *= 5.0
         bits = inputs.f32_to_bf16_bits(qkv)
         ctx = api.pd_attention_fwd(dev_bf16(bits), batch=b2, seq=s2, heads=h2)
-        pick = [0, b2 // 2, b2 - 1]
+        # later work units of a CTA (sequences beyond the first few) are where the two query blocks in flight drift
+        # furthest apart: sample them densely
+        pick = sorted(set([0, b2 - 1] + list(range(b2 // 4, b2, 3))))
         for bb in pick:
             rows = slice(bb * s2, (bb + 1) * s2)
             ref = oracle.attention(inputs.bf16_bits_to_f32(bits[rows]), 1, s2, h2, 64)
