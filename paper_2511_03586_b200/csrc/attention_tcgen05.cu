@@ -5,7 +5,7 @@
 // on the packed projection qkv[tokens, 3*hidden] = [Q | K | V].  Scores and
 // probabilities never leave the SM.
 //
-// One persistent CTA of 416 threads per SM walks over work units of (batch,
+// One persistent CTA of 512 threads per SM walks over work units of (batch,
 // head, pair of 128-query blocks).  K and V of the head (up to 512 x 64 each)
 // sit in shared memory in four chunks of 128 keys, each with its own full and
 // empty barrier, so that the next unit's chunks stream in while the current
@@ -16,14 +16,14 @@
 // tensor memory (all 512 columns), so that the tensor core, the exponential
 // unit and the barrier round trips overlap, also across unit boundaries.
 //
-//   warp 8, one lane : TMA producer (per unit: Q of each slot, then the K and V
+//   warp 8, lane 16  : TMA producer (per unit: Q of each slot, then the K and V
 //                      chunks in the order the previous unit releases them).
-//   warps 9, 11      : score issuers, one thread per slot, each in a warp of
-//                      its own (see kProducerWarp below): for block g of
+//   warps 8, 10      : score issuers, one thread per slot, each in a warp of
+//                      its own (see kScoreWarp0 below): for block g of
 //                      64 keys S = Q K_g^T (128 x 64 x 64) into one of the slot's
 //                      two score buffers, as soon as the softmax warps have
 //                      read that buffer's previous contents.
-//   warps 10, 12     : output issuers, one thread per slot: when the
+//   warps 9, 11      : output issuers, one thread per slot: when the
 //                      slot's softmax warps have published P_g,
 //                      O += P_g V_g (128 x 64 x 64) into the slot's 64 output
 //                      columns, P_g read from tensor memory as the A operand.
@@ -42,10 +42,14 @@
 //                      by 2^(m_old - m_new) through a tensor-memory load / store
 //                      round trip, and the block redone.  O / l is therefore the
 //                      exact softmax for any finite input, and on ordinary
-//                      inputs every score is read once.  Finally the thread
-//                      reads its O row, divides by l and stages 64 bf16 values
-//                      in shared memory, from where each
-//                      warp's 32 rows go to Ctx with one TMA store.
+//                      inputs every score is read once.  At the end of the
+//                      unit the row sums go to the epilogue warps through
+//                      shared memory and the warp moves on to the next unit.
+//   warps 12-15      : epilogue, one thread per query row and both slots in
+//                      turn: when the unit's last product has landed, read the O
+//                      row, divide by l, stage 64 bf16 values in shared memory,
+//                      from where each warp's 32 rows go to Ctx with one TMA
+//                      store; then release O to the next unit's products.
 // Keys beyond the sequence length are zero-filled by TMA and masked out; query
 // rows beyond it are computed and discarded.
 // Every mbarrier wait is bounded (see mbar_wait): on expiry a code is recorded
@@ -63,14 +67,18 @@ constexpr int kBlockQ = 128;      // queries per slot = TMEM lanes
 constexpr int kBlockK = 64;       // keys per score block
 constexpr int kMaxKeys = 512;
 constexpr int kSlots = 2;         // query blocks in flight
-constexpr int kThreads = 416;
-constexpr int kSlotThreads = 128;
-// warps 0-7 softmax; then one warp per single-thread role.  Every tcgen05.mma / tcgen05.commit issuing thread has a
-// warp of its own: two lanes of one warp that reach the same tcgen05 instruction together, with different
-// operands, do not get two independent operations (attention with peaked rows came out wrong that way whenever
-// the two slots drifted apart).
-constexpr int kProducerWarp = 8, kScoreWarp0 = 9, kOutputWarp0 = 10, kScoreWarp1 = 11, kOutputWarp1 = 12;
-constexpr int kAllocWarp = kScoreWarp0;
+constexpr int kThreads = 512;
+constexpr int kSlotThreads = 128, kSlotWarps = kSlotThreads / 32;
+// warps 0-7 softmax, 8-11 the four MMA-issuing threads, 12-15 epilogue (sixteen warps: 128 registers a thread).
+// Every tcgen05.mma / tcgen05.commit issuing thread has a warp of its own: two lanes of one warp that reach the
+// same tcgen05 instruction together, with different operands, do not get two independent operations (attention
+// with peaked rows came out wrong that way whenever the two slots drifted apart).  The TMA producer issues no
+// tcgen05 instruction and rides along as another lane of the first issuer's warp.
+constexpr int kScoreWarp0 = 8, kOutputWarp0 = 9, kScoreWarp1 = 10, kOutputWarp1 = 11;
+constexpr int kProducerWarp = kScoreWarp0, kProducerLane = 16;
+constexpr int kEpilogueWarp0 = 12;  // warp w reads the tensor-memory lanes 32 * (w % 4) ... + 31
+constexpr int kAllocWarp = kOutputWarp0;
+static_assert(kEpilogueWarp0 % 4 == 0 && kThreads == 32 * (kEpilogueWarp0 + 4), "epilogue warps cover the four lane quarters");
 
 constexpr int kSmemK = kMaxKeys * kD * 2;        // 64 KiB
 constexpr int kSmemV = kMaxKeys * kD * 2;        // 64 KiB
@@ -79,8 +87,9 @@ constexpr int kSmemO = kBlockQ * kD * 2;         // 16 KiB of output staging per
 constexpr int kChunkKeys = 128;                  // K and V arrive, and are released, in chunks of 128 keys
 constexpr int kChunks = kMaxKeys / kChunkKeys;
 constexpr int kSmemChunk = kChunkKeys * kD * 2;  // 16 KiB
+constexpr int kSmemL = kSlots * kBlockQ * 4;     // row sums handed from the softmax warps to the epilogue warps
 constexpr int kSmemCtrl = 1024;
-constexpr int kSmemBytes = kSmemK + kSmemV + kSlots * (2 * kSmemQ + kSmemO) + kSmemCtrl + 1024 /*alignment slack*/;
+constexpr int kSmemBytes = kSmemK + kSmemV + kSlots * (2 * kSmemQ + kSmemO) + kSmemL + kSmemCtrl + 1024 /*alignment slack*/;
 
 // tensor-memory columns: score buffer b of slot s at 128*s + 64*b, output accumulator of slot s at 256 + 64*s,
 // probability buffer b of slot s (64 bf16 per row in 32 columns) at 384 + 64*s + 32*b
@@ -129,7 +138,8 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t sK = smem_base, sV = sK + kSmemK, sQ = sV + kSmemV, sO = sQ + kSlots * 2 * kSmemQ;
-  const uint32_t bar_base = sO + kSlots * kSmemO;
+  const uint32_t sL = sO + kSlots * kSmemO;
+  const uint32_t bar_base = sL + kSmemL;
   // barriers (8 bytes each); [c] = chunk of 128 keys, [s] = slot, [s][b] = slot and buffer
   auto k_full = [&](int c) { return bar_base + 8u * c; };
   auto k_empty = [&](int c) { return bar_base + 32u + 8u * c; };
@@ -143,7 +153,8 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   auto s_empty = [&](int s, int b) { return bar_base + 256u + 8u * (2 * s + b); };
   auto p_full = [&](int s, int b) { return bar_base + 288u + 8u * (2 * s + b); };
   auto p_empty = [&](int s, int b) { return bar_base + 320u + 8u * (2 * s + b); };
-  const uint32_t drain_bar = bar_base + 352;  // four of them, one per MMA-issuing thread
+  auto l_full = [&](int s) { return bar_base + 352u + 8u * s; };
+  const uint32_t drain_bar = bar_base + 368;  // four of them, one per MMA-issuing thread
   uint8_t* ctrl = smem_gen + (bar_base - smem_base) + 512;
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(ctrl);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(ctrl + 4);
@@ -156,11 +167,11 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
     }
     for (int i = 0; i < 4; ++i) mbar_init(drain_bar + 8u * i, 1);
     for (int s = 0; s < kSlots; ++s) {
-      mbar_init(o_full(s), 1); mbar_init(o_empty(s), (kSlotThreads / 32));
+      mbar_init(o_full(s), 1); mbar_init(o_empty(s), kSlotWarps); mbar_init(l_full(s), kSlotWarps);
       for (int b = 0; b < 2; ++b) {
         mbar_init(q_full(s, b), 1); mbar_init(q_empty(s, b), 1);
-        mbar_init(s_full(s, b), 1); mbar_init(s_empty(s, b), (kSlotThreads / 32));
-        mbar_init(p_full(s, b), (kSlotThreads / 32)); mbar_init(p_empty(s, b), 1);
+        mbar_init(s_full(s, b), 1); mbar_init(s_empty(s, b), kSlotWarps);
+        mbar_init(p_full(s, b), kSlotWarps); mbar_init(p_empty(s, b), 1);
       }
     }
     *abort_flag = 0;
@@ -191,11 +202,11 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   const int G = p.k_blocks;
   const int NC = (G + 1) >> 1;  // chunks of 128 keys in use; chunk c holds score blocks 2c and 2c + 1
 
-  if (warp == kProducerWarp) {
+  if (warp == kProducerWarp && lane == kProducerLane) {
     // ------------------------------------------------------------- TMA producer
     // Per unit: the two query tiles (into the slot's other buffer, normally free long before), then the chunks
     // of K and V in the order in which the previous unit releases them.
-    if (lane == 0) {
+    {
       prefetch_tensormap(&tmap_q); prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v);
       uint32_t n_unit = 0, n_q[kSlots] = {0, 0};
       uint32_t armed_k = 0, armed_v = 0;  // bit c: chunk c of the current unit has been requested
@@ -339,16 +350,14 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         mbar_wait(drain_bar + 8u * s, 0, &never, nullptr, 0, 20000000ull);
       }
     }
-  } else {
+  } else if (warp < 2 * kSlotWarps) {
     // ------------------------------------------------------------------ softmax
     const int slot = warp >> 2, quarter = warp & 3;
     const int row = quarter * 32 + lane;  // query row within the block = TMEM lane
     const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const uint32_t t_o = t_lane + kTmemO + slot * kD;
-    const uint32_t sw = (uint32_t)(lane & 7);
     uint32_t t = 0, n_us = 0;  // score blocks and units this slot has processed
     bool ok = true;
-    bool store_pending = false;  // this warp's output store may still be reading the staging tile
     for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x) {
       int b, h, qb0, nslots;
       unit_coords(unit, b, h, qb0, nslots);
@@ -494,44 +503,66 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         if (lane == 0) mbar_arrive(p_full(slot, buf));
       }
       if (!ok) break;
-      // ---- output: O / l -> bf16 -> the slot's staging tile -> one TMA store of 32 rows x 128 bytes per
-      // warp; rows beyond the sequence are clipped by the tensor map
-      if (store_pending) {
+      // ---- the row sums go to the epilogue warps, which finish the unit while this warp starts the next one.
+      // The epilogue releases O after it has read the slot's previous sums; with eight blocks a unit that
+      // happened long ago, with one or two this wait is what keeps the hand-over in step.
+      if (!mbar_wait(o_empty(slot), (n_us & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+      ++n_us;
+      st_shared_f32(sL + (uint32_t)(slot * kBlockQ + row) * 4u, l);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(l_full(slot));
+    }
+  } else {
+    // ----------------------------------------------------------------- epilogue
+    // O / l -> bf16 -> the slot's staging tile -> one TMA store of 32 rows x 128 bytes per warp; rows beyond the
+    // sequence are clipped by the tensor map.
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t sw = (uint32_t)(lane & 7);
+    uint32_t n_us[kSlots] = {0, 0};
+    bool ok = true;
+    for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x) {
+      int b, h, qb0, nslots;
+      unit_coords(unit, b, h, qb0, nslots);
+      for (int slot = 0; slot < nslots; ++slot) {
+        const uint32_t ph = n_us[slot] & 1u;
+        ++n_us[slot];
+        if (!mbar_wait(l_full(slot), ph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+        const float inv = 1.0f / ld_shared_f32(sL + (uint32_t)(slot * kBlockQ + row) * 4u);
+        if (!mbar_wait(o_full(slot), ph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
+        tcgen05_fence_after_sync();
+        // this warp's previous stores must have read their staging rows
         if (lane == 0) tma_store_wait_read<0>();
         __syncwarp();
-        store_pending = false;
-      }
-      if (!mbar_wait(o_full(slot), n_us & 1u, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
-      ++n_us;
-      tcgen05_fence_after_sync();
-      const float inv = 1.0f / l;
-      const uint32_t o_row = sO + slot * kSmemO + (uint32_t)row * 128u;
+        const uint32_t t_o = t_lane + kTmemO + slot * kD;
+        const uint32_t o_row = sO + slot * kSmemO + (uint32_t)row * 128u;
 #pragma unroll
-      for (int c0 = 0; c0 < kD; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld_32x32b_x32(t_o + c0, r);
-        tmem_ld_wait();
+        for (int c0 = 0; c0 < kD; c0 += 32) {
+          uint32_t r[32];
+          tmem_ld_32x32b_x32(t_o + c0, r);
+          tmem_ld_wait();
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          uint4 w;
-          w.x = pack_bf16x2(__uint_as_float(r[8 * u]) * inv, __uint_as_float(r[8 * u + 1]) * inv);
-          w.y = pack_bf16x2(__uint_as_float(r[8 * u + 2]) * inv, __uint_as_float(r[8 * u + 3]) * inv);
-          w.z = pack_bf16x2(__uint_as_float(r[8 * u + 4]) * inv, __uint_as_float(r[8 * u + 5]) * inv);
-          w.w = pack_bf16x2(__uint_as_float(r[8 * u + 6]) * inv, __uint_as_float(r[8 * u + 7]) * inv);
-          st_shared_v4(o_row + (((uint32_t)(c0 / 8 + u) ^ sw) << 4), w);
+          for (int u = 0; u < 4; ++u) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(r[8 * u]) * inv, __uint_as_float(r[8 * u + 1]) * inv);
+            w.y = pack_bf16x2(__uint_as_float(r[8 * u + 2]) * inv, __uint_as_float(r[8 * u + 3]) * inv);
+            w.z = pack_bf16x2(__uint_as_float(r[8 * u + 4]) * inv, __uint_as_float(r[8 * u + 5]) * inv);
+            w.w = pack_bf16x2(__uint_as_float(r[8 * u + 6]) * inv, __uint_as_float(r[8 * u + 7]) * inv);
+            st_shared_v4(o_row + (((uint32_t)(c0 / 8 + u) ^ sw) << 4), w);
+          }
+        }
+        // O (and the row sums) have been read: the next unit's products may overwrite them
+        tcgen05_fence_before_sync();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(o_empty(slot));
+          tma_store_4d(&tmap_o, sO + slot * kSmemO + (uint32_t)(quarter * 32) * 128u, 0,
+                       (qb0 + slot) * kBlockQ + quarter * 32, h, b);
+          tma_store_commit();
         }
       }
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) {
-        tma_store_4d(&tmap_o, sO + slot * kSmemO + (uint32_t)(quarter * 32) * 128u, 0,
-                     (qb0 + slot) * kBlockQ + quarter * 32, h, b);
-        tma_store_commit();
-      }
-      store_pending = true;
-      tcgen05_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(o_empty(slot));
     }
     // shared memory must outlive every store that still reads it
     if (lane == 0) tma_store_wait_all<0>();

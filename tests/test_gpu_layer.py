@@ -55,6 +55,21 @@ def test_attention_against_oracle(api, seq):
     assert bool(torch.isfinite(ctx.float()).all())
 
 
+@pytest.mark.parametrize("dims", [(40, 64, 8), (25, 128, 7), (12, 200, 14)])
+def test_attention_many_short_sequences(api, dims):
+    # several work units per CTA with only one to four key blocks each: the hand-over of the row sums from the
+    # softmax warps to the epilogue warps and the reuse of every buffer happen at the shortest possible distance
+    batch, seq, heads = dims
+    rng = np.random.default_rng(seq + heads)
+    qkv = rng.normal(0, 1, size=(batch * seq, 3 * heads * 64)).astype(np.float32)
+    qkv[:, :heads * 64] *= 4.0
+    bits = inputs.f32_to_bf16_bits(qkv)
+    ctx = api.pd_attention_fwd(dev_bf16(bits), batch=batch, seq=seq, heads=heads)
+    ref = oracle.attention(inputs.bf16_bits_to_f32(bits), batch, seq, heads, 64)
+    assert max_rel_floored(host(ctx), ref) < TOL
+    assert api.pd_get_device_status() == 0
+
+
 def test_attention_peaked_rows_and_errors(api):
     # large logits: one key dominates each row; the exact (max-first) softmax must not overflow
     batch, seq, heads = 1, 512, 1
