@@ -97,12 +97,12 @@ constexpr uint32_t kTmemS = 0, kTmemO = 256, kTmemP = 384, kTmemCols = 512;
 
 constexpr float kScale = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
 constexpr float kRescaleThreshold = 16.0f;               // largest exponent of 2 tolerated before m is raised
-// A quarter of the exponentials are evaluated on the FMA pipe (2^a = 2^round(a) * P(a - round(a)), P the degree-3
-// fit printed by fit_exp2_poly.py, relative error 7.5e-5, far below the bf16 rounding of the stored probability),
-// the rest by the special-function unit, which alone would bound the softmax warps; a quarter was the fastest
-// share measured (none: 73.3 us, 1/8: 71.1, 1/4: 70.1, 5/16: 70.6, 1/2: 72.3 for batch 32 x 16 heads x 512).
+// Five sixteenths of the exponentials are evaluated on the FMA pipe (2^a = 2^round(a) * P(a - round(a)), P the
+// degree-3 fit printed by fit_exp2_poly.py, relative error 7.5e-5, far below the bf16 rounding of the stored
+// probability), the rest by the special-function unit, which alone would bound the softmax warps; the fastest
+// share measured (1/8: 65.4 us, 1/4: 64.2, 5/16: 62.7, 3/8: 64.7 for batch 32 x 16 heads x 512, standalone).
 // Bit k of the mask = 1: pair k of each group of sixteen pairs takes the polynomial.
-constexpr uint32_t kPolyPairMask = 0x8888u;
+constexpr uint32_t kPolyPairMask = 0xA888u;
 constexpr float kExp2C0 = 9.999280572e-01f, kExp2C1 = 6.932609677e-01f, kExp2C2 = 2.426111251e-01f,
                 kExp2C3 = 5.517166853e-02f;
 constexpr float kExp2Magic = 12582912.0f;  // 1.5 * 2^23: adding it leaves round(a) in the low mantissa bits
@@ -619,13 +619,8 @@ pd_status launch_fused_attention(const __nv_bfloat16* qkv, __nv_bfloat16* ctx, i
   const int64_t units = batch * heads * p.units_per_head;
   if (units > 0x7fffffff) return PD_ERR_BAD_SHAPE;
   p.num_units = (int)units;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attention_fwd_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kSmemBytes);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_allowed;  // one per kernel (template instantiation)
+  if (pd_status st = allow_dynamic_smem(attention_fwd_tcgen05_kernel, kSmemBytes, smem_allowed); st != PD_OK) return st;
   const int grid = p.num_units < sm_count() ? p.num_units : sm_count();
   launch_pdl(attention_fwd_tcgen05_kernel, dim3(grid), dim3(kThreads), kSmemBytes, s, tq, tk, tv, to, p);
   return check_launch();

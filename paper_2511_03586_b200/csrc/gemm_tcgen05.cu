@@ -237,12 +237,8 @@ pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
   p.alpha = g.alpha; p.c_is_f32 = g.c_dtype == PD_F32; p.act = g.act;
 
   auto kernel = gemm_bf16_tcgen05_kernel<BN, B_NK, C_F32, GATED>;
-  static bool attr_set = false;  // per template instantiation
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_allowed;  // one per kernel (template instantiation)
+  if (pd_status st = allow_dynamic_smem(kernel, C::kSmemBytes, smem_allowed); st != PD_OK) return st;
   const int grid = p.num_tiles < sm_count() ? p.num_tiles : sm_count();
   launch_pdl(kernel, dim3(grid), dim3(kThreads), C::kSmemBytes, s, ta, tb, tb2, tc, p);
   return check_launch();

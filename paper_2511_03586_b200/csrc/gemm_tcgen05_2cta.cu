@@ -215,12 +215,8 @@ pd_status launch_pair_variant(const GemmProblem& g, cudaStream_t s) {
   p.alpha = g.alpha; p.c_is_f32 = C_F32; p.act = g.act;
 
   auto kernel = gemm_bf16_tcgen05_pair_kernel<B_NK, C_F32>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_allowed;  // one per kernel (template instantiation)
+  if (pd_status st = allow_dynamic_smem(kernel, kSmemBytes, smem_allowed); st != PD_OK) return st;
   const int pairs = (int)(tiles < sm_count() / 2 ? tiles : sm_count() / 2);
   launch_pdl(kernel, dim3(2 * pairs), dim3(kThreads), kSmemBytes, s, ta, tb, tc, p);
   return check_launch();

@@ -418,12 +418,8 @@ pd_status launch_ln_variant(const GemmProblem& g, const float* gamma, const floa
   LnParams ln{gamma, beta, eps, p.tiles_n};
 
   auto kernel = gemm_bias_residual_layernorm_kernel<B_NK>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_allowed;  // one per kernel (template instantiation)
+  if (pd_status st = allow_dynamic_smem(kernel, kSmemBytes, smem_allowed); st != PD_OK) return st;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((sm_count() / ln.cluster) * ln.cluster);
   cfg.blockDim = dim3(kLnThreads);

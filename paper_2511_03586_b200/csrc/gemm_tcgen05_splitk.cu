@@ -324,12 +324,8 @@ pd_status launch_split_variant(const GemmProblem& g, cudaStream_t s) {
   SplitParams sp{p.c_is_f32, g.residual};
 
   auto kernel = gemm_bf16_splitk_cluster_kernel<BN, B_NK, GATED, S>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes);
-    if (e != cudaSuccess) return record_cuda_error(e);
-    attr_set = true;
-  }
+  static PerDeviceFlag smem_allowed;  // one per kernel (template instantiation)
+  if (pd_status st = allow_dynamic_smem(kernel, C::kSmemBytes, smem_allowed); st != PD_OK) return st;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p.num_tiles * split);
   cfg.blockDim = dim3(kThreads);

@@ -23,6 +23,26 @@ int sm_count();
 // Device address of the status word the bounded waits report to (nullptr on failure).
 int* device_status_ptr();
 
+// Raises the dynamic shared-memory limit of `kernel` on the current device, once per device (the attribute belongs
+// to the device's context, and one process may drive several devices).  `done` is the caller's per-kernel record.
+constexpr int kMaxDevicesPerProcess = 64;
+struct PerDeviceFlag {
+  bool set[kMaxDevicesPerProcess] = {};
+};
+template <typename Kernel>
+inline pd_status allow_dynamic_smem(Kernel kernel, int bytes, PerDeviceFlag& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return record_cuda_error(e);
+  if (dev < 0 || dev >= kMaxDevicesPerProcess) return PD_ERR_UNSUPPORTED;
+  if (!done.set[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return record_cuda_error(e);
+    done.set[dev] = true;
+  }
+  return PD_OK;
+}
+
 // Launch with programmatic stream serialisation: the kernel may become resident and run its prologue while the
 // previous kernel of the stream is still draining; it must call griddep_wait() before it touches global memory
 // that an earlier kernel may still read or write.  Kernels call griddep_launch_dependents() to let their own
