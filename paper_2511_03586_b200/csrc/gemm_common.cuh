@@ -117,7 +117,7 @@ struct ResidualRegs {
 // or 32 fp32 columns (one step).  The two warps of a lane group take alternate
 // chunks.  `first_tile`/`tile_stride` enumerate the tiles, `row_block` maps a
 // tile's m index to the first of the 128 rows held in this CTA's tensor memory,
-// `release` is called once per tile after the warp's last tensor-memory read.
+// `release` is called once per tile by one lane, after the whole warp's last tensor-memory read.
 template <int BN, bool C_F32, typename RowBlockFn, typename ReleaseFn>
 __device__ __forceinline__ void epilogue_warp(const KernelParams& p, const CUtensorMap* tmap_c, uint32_t tmem_base,
                                               uint32_t epi_base, uint32_t acc_full_bar0, volatile int* abort_flag,
@@ -239,7 +239,8 @@ __device__ __forceinline__ void epilogue_warp(const KernelParams& p, const CUten
       cur = nxt;
     }
     tcgen05_fence_before_sync();
-    release(acc);
+    __syncwarp();
+    if (lane == 0) release(acc);  // one arrival per warp
   }
   // Shared memory must outlive every store that still reads it.
   if (lane == 0) tma_store_wait_all<0>();
@@ -319,7 +320,8 @@ __device__ __forceinline__ void epilogue_warp_gated(const KernelParams& p, const
       ++stores;
     }
     tcgen05_fence_before_sync();
-    release(acc);
+    __syncwarp();
+    if (lane == 0) release(acc);  // one arrival per warp
   }
   if (lane == 0) tma_store_wait_all<0>();
   __syncwarp();

@@ -71,7 +71,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(acc_full_bar(a), 1);
-      mbar_init(acc_empty_bar(a), 2 * kEpilogueThreads);  // both CTAs' epilogue threads; used in the even CTA only
+      mbar_init(acc_empty_bar(a), 2 * kEpilogueThreads / 32);  // both CTAs' epilogue warps; used in the even CTA only
     }
     mbar_init(drain_bar, 1);
     *abort_flag = 0;
