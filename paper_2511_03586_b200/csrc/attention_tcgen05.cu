@@ -194,7 +194,9 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   auto unit_coords = [&](int unit, int& b, int& h, int& qb0, int& nslots) {
     const int per_bh = p.units_per_head;
     const int bh = unit / per_bh;
-    b = bh / p.heads;
+    // last sequence first: inside the layer the projection before this kernel wrote qkv first row first, and what it
+    // wrote last is what is still in L2
+    b = p.batch - 1 - bh / p.heads;
     h = bh % p.heads;
     qb0 = (unit % per_bh) * kSlots;
     nslots = min(kSlots, p.q_blocks - qb0);

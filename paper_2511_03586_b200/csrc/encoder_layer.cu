@@ -181,6 +181,8 @@ pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_we
     g.bias = w->b_ffn2; g.residual = h1; g.ldr = H;
     if (fuse_ln) {
       g.C = y;
+      // Mid (T x F bf16) exceeds L2 at the configured size and FFN-up wrote it first row first
+      g.rows_descending = true;
       st = launch_gemm_layernorm(g, w->ln2_gamma, w->ln2_beta, desc->ln_eps, stream);
       mark();
     } else {

@@ -59,6 +59,7 @@ struct LnParams {
   const float* beta;
   float eps;
   int cluster;  // CTAs per cluster = N / 256
+  int descending;  // walk the row blocks from the last to the first (GemmProblem::rows_descending)
 };
 
 enum : int { kTimeoutLnStats = 105, kTimeoutLnPair = 106, kTimeoutLnConsumed = 107 };
@@ -94,6 +95,8 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
   const int nt = (int)cluster_ctarank();            // this CTA's column tile
   const int cluster_id = blockIdx.x / ln.cluster;
   const int num_clusters = gridDim.x / ln.cluster;  // row blocks are dealt round-robin to clusters
+  // step i of a cluster works on row block phys(cluster_id + i * num_clusters)
+  auto phys = [&](int lt) { return ln.descending ? p.tiles_m - 1 - lt : lt; };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -130,7 +133,8 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
       prefetch_tensormap(&tmap_b);
       uint32_t it = 0;
       bool ok = true;
-      for (int mt = cluster_id; mt < p.tiles_m && ok; mt += num_clusters) {
+      for (int lt = cluster_id; lt < p.tiles_m && ok; lt += num_clusters) {
+        const int mt = phys(lt);
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
@@ -164,7 +168,7 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
       uint32_t it = 0;
       int local = 0;
       bool ok = true;
-      for (int mt = cluster_id; mt < p.tiles_m && ok; mt += num_clusters, ++local) {
+      for (int lt = cluster_id; lt < p.tiles_m && ok; lt += num_clusters, ++local) {
         const int acc = local & 1;
         const uint32_t acc_ph = (local >> 1) & 1u;
         if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc)) { ok = false; break; }
@@ -216,9 +220,9 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
 
     // The residual of this thread's 64 columns of one row, fetched one tile ahead of its use.
     uint4 res[4][2];
-    auto load_residual = [&](int mt) {
-      const int m = mt * BM + row;
-      if (p.residual == nullptr || mt >= p.tiles_m || m >= p.M) return;
+    auto load_residual = [&](int lt) {
+      const int m = phys(lt) * BM + row;
+      if (p.residual == nullptr || lt >= p.tiles_m || m >= p.M) return;
       const uint4* rr = reinterpret_cast<const uint4*>(p.residual + (int64_t)m * p.ldr + n_tile + c_base);
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -231,7 +235,8 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     int local = 0;
     if (lane == 0) prefetch_tensormap(&tmap_c);
     load_residual(cluster_id);
-    for (int mt = cluster_id; mt < p.tiles_m; mt += num_clusters, ++local) {
+    for (int lt = cluster_id; lt < p.tiles_m; lt += num_clusters, ++local) {
+      const int mt = phys(lt);
       const int acc = local & 1;
       const uint32_t acc_ph = (local >> 1) & 1u;
       const uint32_t tile_ph = local & 1u;  // phase parity of the once-per-tile barriers
@@ -239,8 +244,8 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
       // the previous tile's phase of stats_bar is complete (this warp waited for it): expect this tile's bytes
       if (warp == 2 && lane == 0) mbar_arrive_expect_tx(stats_bar, (uint32_t)ln.cluster * BM * 8u);
       // the next tile's residual (one 128-byte line per thread) starts its way from DRAM into L2 a tile ahead
-      if (p.residual != nullptr && mt + num_clusters < p.tiles_m && (mt + num_clusters) * BM + row < p.M)
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(p.residual + ((int64_t)(mt + num_clusters) * BM + row) * p.ldr +
+      if (p.residual != nullptr && lt + num_clusters < p.tiles_m && phys(lt + num_clusters) * BM + row < p.M)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(p.residual + ((int64_t)phys(lt + num_clusters) * BM + row) * p.ldr +
                                                       n_tile + c_base));
       if (!mbar_wait(acc_full_bar(acc), acc_ph, abort_flag, p.status, kTimeoutEpilogue)) break;
       tcgen05_fence_after_sync();
@@ -285,7 +290,7 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
           a2[j & 1] = fma_f32x2(d, d, a2[j & 1]);
         }
       }
-      load_residual(mt + num_clusters);  // the next tile's residual travels during the exchange and pass 2
+      load_residual(lt + num_clusters);  // the next tile's residual travels during the exchange and pass 2
       float mean_p, m2_p;  // of this thread's 64 values
       {
         float s1a, s1b, s2a, s2b;
@@ -415,7 +420,7 @@ pd_status launch_ln_variant(const GemmProblem& g, const float* gamma, const floa
   p.batch_inner = 1;
   p.num_tiles = p.tiles_m * p.tiles_n;
   p.alpha = g.alpha; p.c_is_f32 = 0; p.act = 0;
-  LnParams ln{gamma, beta, eps, p.tiles_n};
+  LnParams ln{gamma, beta, eps, p.tiles_n, g.rows_descending ? 1 : 0};
 
   auto kernel = gemm_bias_residual_layernorm_kernel<B_NK>;
   static PerDeviceFlag smem_allowed;  // one per kernel (template instantiation)

@@ -226,6 +226,10 @@ struct GemmProblem {
   const void* B2 = nullptr;                  // bf16 [K, N], row stride ldb: second weight of the gated form, or null
   const __nv_bfloat16* residual = nullptr;   // bf16 [M, N], row stride ldr, or null (unbatched only)
   int64_t ldr = 0;
+  // Walk the row blocks of C from the last to the first (LayerNorm GEMM only).  A consumer whose A operand is
+  // larger than L2 and was written first row first by the launch before it finds the most recently written
+  // rows still in L2 when it starts at the far end; results do not depend on the order.
+  bool rows_descending = false;
 };
 pd_status launch_gemm(const GemmProblem& p, cudaStream_t s);
 // The same contraction on 256 x 256 tiles computed by pairs of CTAs (cta_group::2).
