@@ -32,7 +32,7 @@
 //                      thread cost more than the products themselves.)
 //   warps 0-3, 4-7   : softmax of slot 0 / slot 1, one thread per query row.
 //                      The row keeps a reference exponent m (the maximum of its
-//                      first block).  For each block it forms
+//                      first 32 scores).  For each block it forms
 //                      p = 2^(s * log2(e) / 8 - m) from the scores in tensor
 //                      memory, adds them to the fp32 row sum l, releases the
 //                      score buffer and writes P as bf16 into the probability
@@ -373,30 +373,17 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         const int key0 = g * kBlockK;
         if (!mbar_wait(s_full(slot, buf), use_ph, abort_flag, p.status, kTimeoutAttnSoftmax)) { ok = false; break; }
         tcgen05_fence_after_sync();
-        if (g == 0) {
-          // the first block fixes the reference: its maximum
-          float bm = -INFINITY;
-#pragma unroll
-          for (int cc = 0; cc < kBlockK / 32; ++cc) {
-            uint32_t r[32];
-            tmem_ld_32x32b_x32(t_s + cc * 32, r);
-            tmem_ld_wait();
-            const int c0 = key0 + cc * 32;
-            float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (c0 + i < p.seq) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(r[i]));
-            bm = fmaxf(bm, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
-          }
-          mk = bm * kScale;
-        }
         // exponentials of the block against reference `ref`: fills pk and returns the row's partial sum
         // (two fp32 values per instruction where the operation exists in packed form)
         uint32_t pk[kBlockK / 2];  // the block's probabilities, two bf16 per register
-        auto exp_block = [&](float ref) {
+        // `first`: the unit's first block, which also fixes the row's reference exponent: the maximum of the first
+        // 32 scores, taken from the registers the exponentials are about to use (no second pass over the block).
+        // Any reference that is attained by some key keeps l >= 1; the check below covers the rest.
+        auto exp_block = [&](float ref, bool first) {
           uint64_t part2[2] = {0, 0};
           float part = 0.f;
-          const uint64_t scale2 = pack_f32x2(kScale, kScale), nref2 = pack_f32x2(-ref, -ref);
+          const uint64_t scale2 = pack_f32x2(kScale, kScale);
+          uint64_t nref2 = pack_f32x2(-ref, -ref);
           uint32_t r[2][32];
           tmem_ld_32x32b_x32(t_s, r[0]);
 #pragma unroll
@@ -405,6 +392,15 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
             if (cc + 1 < kBlockK / 32) tmem_ld_32x32b_x32(t_s + (cc + 1) * 32, r[(cc & 1) ^ 1]);
             const uint32_t(&rr)[32] = r[cc & 1];
             const int c0 = key0 + cc * 32;
+            if (first && cc == 0) {
+              float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (c0 + i < p.seq) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(rr[i]));
+              ref = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * kScale;
+              mk = ref;
+              nref2 = pack_f32x2(-ref, -ref);
+            }
             if (c0 + 32 <= p.seq) {
 #pragma unroll
               for (int i = 0; i < 32; i += 2) {
@@ -462,7 +458,7 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
           }
           return amax;
         };
-        float part = exp_block(mk);
+        float part = exp_block(mk, g == 0);
         // A term above 2^16 shows in the sum, so the sum alone clears the ordinary case; !(<=) also catches NaN.
         if (__any_sync(0xffffffffu, !(part <= kRescaleSum))) {
           // rare: this block towers over the reference.  Raise the reference of the rows concerned, rescale
@@ -487,7 +483,7 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
             tmem_st_wait();
           }
           if (raise) mk += amax;
-          part = exp_block(mk);
+          part = exp_block(mk, false);
         }
         l += part;
         // the scores have been read for good: the buffer may take the block after next
