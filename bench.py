@@ -251,6 +251,12 @@ def ops_suite(torch, api, peaks, only: str = ""):
         iters = max(20, min(2000, int(3e9 / (rows * cols * 8))))
         ms = time_launches(torch, lambda i: api.pd_layernorm(xs[i % n], g, b, 1e-5, ys[i % n]), iters)
         rowop_entry(f"layernorm_{rows}x{cols}", ms, rows * cols * 8 + cols * 8, note)
+        if rows * cols * 8 <= (32 << 20):
+            # what a plain device copy of the same bytes reaches in the same harness: the ceiling at this size,
+            # where a launch lasts a few microseconds and its ramp-up and tail no longer vanish
+            ms = time_launches(torch, lambda i: ys[i % n].copy_(xs[i % n]), iters)
+            rowop_entry(f"context_copy_{rows}x{cols}", ms, rows * cols * 8,
+                        "torch copy_ of the same bytes, for context: not part of the library")
         del xs, ys
 
     rows, cols = 3072, 4096

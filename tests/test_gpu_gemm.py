@@ -107,6 +107,46 @@ def test_batched_paper_bmm_shape(api, b_is_nk):
     assert np.array_equal(host(c), a64 @ b64)
 
 
+@pytest.mark.parametrize("shape", [(2560, 2048, 128), (2500, 1992, 72), (2304, 2304, 64)])
+def test_partly_filled_last_round_is_exact(api, shape):
+    # 80, 80 and 81 tiles of 256 x 256 on 74 CTA pairs: a second round that only a few pairs take part in, with
+    # ragged right and bottom edges in the second shape; integer inputs, so bit equality
+    M, N, K = shape
+    p = inputs.gemm_integer_inputs(M, N, K, seed=M + N + K, b_is_nk=False)
+    a, b = dev_bf16(p["a_bits"][0]), dev_bf16(p["b_bits"][0])
+    c = Guarded((M, N), torch.float32)
+    api.pd_gemm_bf16(a, b, c.t)
+    torch.cuda.synchronize()
+    c.check()
+    ref = _oracle(p, False)[0]
+    assert np.array_equal(host(c.t), ref)
+    cb = Guarded((M, N), torch.bfloat16)
+    api.pd_gemm_bf16(a, b, cb.t)
+    torch.cuda.synchronize()
+    cb.check()
+    ref_bf16 = inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(ref.astype(np.float32)))
+    assert np.array_equal(host(cb.t), ref_bf16.astype(np.float64))
+
+
+def test_layer_qkv_shape_sampled_rows(api):
+    # the layer's QKV projection: 768 pair tiles = 10 rounds of 74 and 28 left over
+    M, K, N = 16384, 1024, 3072
+    p = inputs.gemm_inputs(M, N, K, seed=7)
+    a, b = dev_bf16(p["a_bits"][0]), dev_bf16(p["b_bits"][0])
+    c32 = api.pd_gemm_bf16(a, b, c_dtype=torch.float32)
+    c = api.pd_gemm_bf16(a, b)
+    # the last round holds the rows from 15872 on: sample there densely and elsewhere sparsely
+    rng = np.random.default_rng(1)
+    pick = np.unique(np.concatenate([[0, 255, 256, M - 1, M - 256, M - 257], rng.integers(0, M, 30),
+                                     rng.integers(M - 768, M, 50)]))
+    ref = oracle.gemm(p["a"][0][pick], p["b"][0])
+    idx = torch.from_numpy(pick).cuda()
+    assert max_rel_floored(host(c32[idx]), ref) < 1e-5
+    assert max_rel_floored(host(c[idx]), ref) < TOL
+    assert bool(torch.isfinite(c32).all())
+    assert torch.equal(c, c32.to(torch.bfloat16))
+
+
 def test_paper_matmul_shape(api):
     M, K, N = 768, 1024, 1024
     p = inputs.gemm_inputs(M, N, K, seed=4)
