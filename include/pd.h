@@ -194,8 +194,10 @@ pd_status pd_set_gemm_split_k(int mode);
  * head h in columns 64h..64h+63 of each block, token t = b*seq + s.
  *   ctx[b, :, 64h..64h+63] = softmax(Q[b,h] K[b,h]^T / 8) V[b,h]
  * ctx: bf16 [batch*seq, heads*64]; must not overlap qkv.  Head dimension is 64
- * and 1 <= seq <= 512 (else PD_ERR_UNSUPPORTED).  Softmax is exact (maximum
- * taken before any exponential) in fp32; probabilities are rounded to bf16 for
+ * and 1 <= seq <= 512 (else PD_ERR_UNSUPPORTED).  Softmax is exact for any
+ * finite input and computed in fp32: every row is referred to a running
+ * reference exponent that is raised, with what has been accumulated rescaled,
+ * before an exponential could overflow.  Probabilities are rounded to bf16 for
  * the second product, which accumulates in fp32. */
 pd_status pd_attention_fwd(const void* qkv, void* ctx, int64_t batch, int64_t seq, int64_t heads,
                            cudaStream_t stream);
