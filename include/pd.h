@@ -12,7 +12,18 @@
  *    and keeps no pointer after it returns.
  *  - Tensors are dense and row-major.  Sizes are in elements, strides (ld*) too.
  *  - Calls validate their arguments on the host, enqueue work on `stream` and
- *    return without synchronising.  On any error nothing has been enqueued.
+ *    return without synchronising.  On an argument error (every status but
+ *    PD_ERR_CUDA) nothing has been enqueued.  The single-kernel entry points
+ *    enqueue nothing on PD_ERR_CUDA either; the chained ones
+ *    (pd_encoder_layer_fwd and its variants, pd_encoder_stack_fwd) stop at the
+ *    launch that failed, with earlier kernels already on the stream: after
+ *    PD_ERR_CUDA from them, y and the workspace hold unspecified values.
+ *  - PD_OK means "enqueued".  The tensor-core entry points (pd_gemm_*,
+ *    pd_swiglu_gemm, pd_attention_fwd, the layer and stack calls) bound every
+ *    wait inside their kernels; a kernel whose wait ran out returns early and
+ *    leaves a code in the device status word, so their results are valid only
+ *    if pd_get_device_status reports 0 after the stream has been synchronised.
+ *    The word is shared by all streams of the device.
  *  - A zero outer extent (rows == 0, M == 0, N == 0, batch == 0) is PD_OK and
  *    launches nothing; a zero reduction extent (cols == 0, K == 0) is
  *    PD_ERR_BAD_SHAPE.
@@ -106,7 +117,10 @@ pd_status pd_bias_gelu_residual(const float* x, const float* bias, const float* 
  * multiples of 8 elements; ldc * sizeof(C element) and strideC * sizeof(C
  * element) multiples of 16 bytes (else PD_ERR_ALIGNMENT); ld* at least the
  * row length; M, N, K otherwise arbitrary (ragged edges are zero-filled on load
- * and clipped on store).  C must not overlap A or B. */
+ * and clipped on store: nothing beyond column N - 1 of a row of C is written,
+ * also when ldc > N; a row end that does not fall on a 16-byte boundary is
+ * written with plain stores instead of a bulk tensor store).  C must not
+ * overlap A or B. */
 pd_status pd_gemm_bf16(const void* A, const void* B, void* C, int64_t M, int64_t N, int64_t K,
                        int64_t lda, int64_t ldb, int64_t ldc, int b_is_nk, pd_dtype c_dtype,
                        int64_t batch, int64_t strideA, int64_t strideB, int64_t strideC,
@@ -226,6 +240,21 @@ typedef struct {
  * `desc` (0 if desc is NULL or invalid). */
 size_t pd_encoder_layer_workspace_bytes(const pd_encoder_layer_desc* desc);
 
+/* Where the intermediates of pd_encoder_layer_fwd live inside its workspace, for
+ * callers that want to inspect them (the stage-by-stage validation of the
+ * paper's Section 2.2 "Transformations": every transformed program is compared
+ * with the original).  offsets[i] and sizes[i] (host arrays of
+ * PD_LAYER_BUFFER_COUNT entries, bytes) describe buffer i under the current
+ * fusion mode; a buffer the layer does not materialise for `desc` has size 0.
+ *   PD_LAYER_BUF_QKV    bf16 [tokens, 3*hidden]     PD_LAYER_BUF_CTX  bf16 [tokens, hidden]
+ *   PD_LAYER_BUF_SCORES fp32 [batch*heads*seq, seq] PD_LAYER_BUF_PRE  fp32 [tokens, hidden]
+ *   PD_LAYER_BUF_PROBS  bf16 [batch*heads*seq, seq] PD_LAYER_BUF_H1   bf16 [tokens, hidden]
+ *                                                   PD_LAYER_BUF_MID  bf16 [tokens, ffn]
+ * NULL arguments: PD_ERR_NULL_POINTER; desc as for pd_encoder_layer_fwd. */
+enum { PD_LAYER_BUF_QKV = 0, PD_LAYER_BUF_SCORES, PD_LAYER_BUF_PROBS, PD_LAYER_BUF_CTX, PD_LAYER_BUF_PRE,
+       PD_LAYER_BUF_H1, PD_LAYER_BUF_MID, PD_LAYER_BUFFER_COUNT };
+pd_status pd_encoder_layer_workspace_layout(const pd_encoder_layer_desc* desc, size_t* offsets, size_t* sizes);
+
 /* Forward pass of one encoder layer, no dropout, no mask, token t = b*seq + s:
  *   QKV = X Wqkv + bqkv
  *   Ctx[b,h] = softmax(Q[b,h] K[b,h]^T / sqrt(64)) V[b,h]
@@ -283,7 +312,8 @@ pd_status pd_set_layernorm_fusion(int mode);
  * = 32 MiB inside the library's device image (held by every GPU that loads the
  * library, until the process exits) instead of a caller-provided workspace.
  *  - Same arguments, results and error codes as pd_encoder_layer_fwd, minus the
- *    workspace.  A shape whose intermediates need more than the array holds
+ *    workspace, checked in the same order (the size check below stands where
+ *    that call checks its workspace).  A shape whose intermediates need more than the array holds
  *    (pd_encoder_layer_workspace_bytes(desc) > 32 MiB; BERT-large fits up to
  *    about 1800 tokens, 1400 with the LayerNorms unfused) is rejected with
  *    PD_ERR_WORKSPACE_TOO_SMALL and nothing is enqueued.
@@ -291,7 +321,8 @@ pd_status pd_set_layernorm_fusion(int mode);
  *    library routine, on any call.
  *  - The first call on each device looks up the array's device address
  *    (cudaGetSymbolAddress, with that device current).  Make that first call
- *    before starting any stream capture.
+ *    before starting any stream capture.  Several host threads may make it at
+ *    once (they store the same address).
  *  - All calls share the one array and it keeps whatever the previous call left
  *    there (every intermediate is fully rewritten before it is read, so nothing
  *    needs clearing).  Two calls that overlap on the GPU - different streams, or

@@ -23,7 +23,7 @@ PD_BF16, PD_F32 = 0, 1
 EXPORTS = (
     "pd_status_string", "pd_last_cuda_error", "pd_get_device_status", "pd_clear_device_status",
     "pd_softmax", "pd_layernorm", "pd_rmsnorm", "pd_bias_gelu_residual", "pd_gemm_bf16", "pd_set_gemm_tile_mode", "pd_attention_fwd",
-    "pd_encoder_layer_workspace_bytes", "pd_encoder_layer_fwd", "pd_encoder_layer_stage_count",
+    "pd_encoder_layer_workspace_bytes", "pd_encoder_layer_workspace_layout", "pd_encoder_layer_fwd", "pd_encoder_layer_stage_count",
     "pd_encoder_layer_stage_name", "pd_encoder_layer_fwd_profiled", "pd_encoder_layer_static_scratch_bytes",
     "pd_encoder_layer_fwd_static",
 )
@@ -76,6 +76,9 @@ def _load() -> ctypes.CDLL:
     lib.pd_attention_fwd.argtypes = [vp, vp, i64, i64, i64, vp]; lib.pd_attention_fwd.restype = st
     lib.pd_encoder_layer_workspace_bytes.argtypes = [ctypes.POINTER(EncoderLayerDesc)]
     lib.pd_encoder_layer_workspace_bytes.restype = ctypes.c_size_t
+    lib.pd_encoder_layer_workspace_layout.argtypes = [ctypes.POINTER(EncoderLayerDesc),
+                                                      ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+    lib.pd_encoder_layer_workspace_layout.restype = st
     lib.pd_encoder_layer_fwd.argtypes = [ctypes.POINTER(EncoderLayerDesc), ctypes.POINTER(EncoderLayerWeights),
                                          vp, vp, vp, ctypes.c_size_t, vp]
     lib.pd_encoder_layer_fwd.restype = st
@@ -297,6 +300,19 @@ def pd_encoder_layer_workspace_bytes(batch: int, seq: int, hidden: int, heads: i
                                      ln_eps: float = 1e-5) -> int:
     d = EncoderLayerDesc(batch, seq, hidden, heads, ffn, ln_eps)
     return int(_lib.pd_encoder_layer_workspace_bytes(ctypes.byref(d)))
+
+
+LAYER_BUFFERS = ("qkv", "scores", "probs", "ctx", "pre", "h1", "mid")
+
+
+def pd_encoder_layer_workspace_layout(batch: int, seq: int, hidden: int, heads: int, ffn: int,
+                                      ln_eps: float = 1e-5) -> dict:
+    """{buffer name: (byte offset, byte size)} of the layer's intermediates inside its workspace."""
+    d = EncoderLayerDesc(batch, seq, hidden, heads, ffn, ln_eps)
+    n = len(LAYER_BUFFERS)
+    off, size = (ctypes.c_size_t * n)(), (ctypes.c_size_t * n)()
+    _check(_lib.pd_encoder_layer_workspace_layout(ctypes.byref(d), off, size), "pd_encoder_layer_workspace_layout")
+    return {name: (int(off[i]), int(size[i])) for i, name in enumerate(LAYER_BUFFERS)}
 
 
 def pd_encoder_layer_fwd(params: EncoderLayerParams, x: torch.Tensor, *, batch: int, seq: int, heads: int,

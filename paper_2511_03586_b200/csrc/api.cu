@@ -1,4 +1,6 @@
 // Status handling, device checks and the device status word of the pd library.
+#include <atomic>
+
 #include "pd_common.cuh"
 
 namespace pd {
@@ -19,42 +21,47 @@ pd_status record_cuda_error(cudaError_t e) {
 }
 
 pd_status require_sm100() {
-  static int cached_major[kMaxDevices];  // 0 = not queried yet
+  // The per-device caches of this file are atomics: concurrent first calls from several host threads each
+  // query the device and store the same value.
+  static std::atomic<int> cached_major[kMaxDevices];  // 0 = not queried yet
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return record_cuda_error(e);
   if (dev < 0 || dev >= kMaxDevices) return PD_ERR_UNSUPPORTED;
-  if (cached_major[dev] == 0) {
-    int major = 0;
+  int major = cached_major[dev].load(std::memory_order_relaxed);
+  if (major == 0) {
     e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
     if (e != cudaSuccess) return record_cuda_error(e);
-    cached_major[dev] = major > 0 ? major : -1;
+    major = major > 0 ? major : -1;
+    cached_major[dev].store(major, std::memory_order_relaxed);
   }
-  return cached_major[dev] == 10 ? PD_OK : PD_ERR_UNSUPPORTED;
+  return major == 10 ? PD_OK : PD_ERR_UNSUPPORTED;
 }
 
 int sm_count() {
-  static int cached[kMaxDevices];
+  static std::atomic<int> cached[kMaxDevices];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 148;
-  if (cached[dev] == 0) {
-    int n = 0;
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
     if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-    cached[dev] = n;
+    cached[dev].store(n, std::memory_order_relaxed);
   }
-  return cached[dev];
+  return n;
 }
 
 int* device_status_ptr() {
-  static int* cached[kMaxDevices];
+  static std::atomic<int*> cached[kMaxDevices];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-  if (!cached[dev]) {
+  int* q = cached[dev].load(std::memory_order_acquire);
+  if (!q) {
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
-    cached[dev] = static_cast<int*>(p);
+    q = static_cast<int*>(p);
+    cached[dev].store(q, std::memory_order_release);
   }
-  return cached[dev];
+  return q;
 }
 
 }  // namespace pd

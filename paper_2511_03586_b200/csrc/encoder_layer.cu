@@ -9,6 +9,8 @@
 //   Y   = LayerNorm(Mid W2 + b2 + H1)                     (GEMM with bias + residual + LayerNorm epilogue)
 // When the hidden size does not suit the fused LayerNorm epilogue (or it is switched off), the two
 // LayerNorm GEMMs write their fp32 sum to a scratch tensor and the LayerNorm row kernel follows.
+#include <atomic>
+
 #include "pd_common.cuh"
 
 namespace pd {
@@ -26,6 +28,7 @@ struct Workspace {
 bool valid_desc(const pd_encoder_layer_desc* d) {
   if (!d) return false;
   if (d->batch < 0 || d->seq <= 0 || d->hidden <= 0 || d->heads <= 0 || d->ffn <= 0) return false;
+  if ((int64_t)d->batch * d->seq > 0x7fffffff) return false;  // the launchers index tokens with int
   if (!(d->ln_eps >= 0.f)) return false;
   return true;
 }
@@ -72,6 +75,20 @@ extern "C" size_t pd_encoder_layer_workspace_bytes(const pd_encoder_layer_desc* 
   return pd::plan(desc).total;
 }
 
+extern "C" pd_status pd_encoder_layer_workspace_layout(const pd_encoder_layer_desc* desc, size_t* offsets,
+                                                       size_t* sizes) {
+  if (!desc || !offsets || !sizes) return PD_ERR_NULL_POINTER;
+  if (!pd::valid_desc(desc)) return PD_ERR_BAD_SHAPE;
+  if (!pd::supported_desc(desc)) return PD_ERR_UNSUPPORTED;
+  const pd::Workspace w = pd::plan(desc);
+  const size_t off[PD_LAYER_BUFFER_COUNT + 1] = {w.qkv, w.scores, w.probs, w.ctx, w.pre, w.h1, w.mid, w.total};
+  for (int i = 0; i < PD_LAYER_BUFFER_COUNT; ++i) {
+    offsets[i] = off[i];
+    sizes[i] = off[i + 1] - off[i];  // the buffers follow one another in this order
+  }
+  return PD_OK;
+}
+
 namespace pd {
 namespace {
 
@@ -79,15 +96,9 @@ constexpr int kStages = 7;
 const char* const kStageNames[kStages] = {"qkv_gemm", "attention", "out_proj_gemm", "layernorm1",
                                           "ffn_up_gemm", "ffn_down_gemm", "layernorm2"};
 
-// Enqueues the whole layer.  When `ev` is not null it holds kStages + 1 events:
-// ev[i] is recorded before stage i and ev[kStages] after the last one.
-pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* w, const void* x, void* y,
-                    void* workspace, size_t workspace_bytes, cudaStream_t stream, cudaEvent_t* ev) {
-  int stage = 0;
-  auto mark = [&]() {
-    if (ev) cudaEventRecord(ev[stage], stream);
-    ++stage;
-  };
+// Argument checks shared by every layer entry point: null pointers, then the shape, then alignment.
+pd_status check_layer_args(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* w, const void* x,
+                           const void* y) {
   if (!desc || !w || !x || !y) return PD_ERR_NULL_POINTER;
   if (!w->w_qkv || !w->w_o || !w->w_ffn1 || !w->w_ffn2 || !w->b_qkv || !w->b_o || !w->b_ffn1 || !w->b_ffn2 ||
       !w->ln1_gamma || !w->ln1_beta || !w->ln2_gamma || !w->ln2_beta)
@@ -98,6 +109,19 @@ pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_we
                         w->ln1_gamma, w->ln1_beta, w->ln2_gamma, w->ln2_beta};
   for (const void* p : ptrs)
     if (!aligned16(p)) return PD_ERR_ALIGNMENT;
+  return PD_OK;
+}
+
+// Enqueues the whole layer.  When `ev` is not null it holds kStages + 1 events:
+// ev[i] is recorded before stage i and ev[kStages] after the last one.
+pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* w, const void* x, void* y,
+                    void* workspace, size_t workspace_bytes, cudaStream_t stream, cudaEvent_t* ev) {
+  int stage = 0;
+  auto mark = [&]() {
+    if (ev) cudaEventRecord(ev[stage], stream);
+    ++stage;
+  };
+  if (pd_status st0 = check_layer_args(desc, w, x, y); st0 != PD_OK) return st0;
   if (desc->batch == 0) return PD_OK;
   const Workspace ws = plan(desc);
   if (!workspace) return PD_ERR_NULL_POINTER;
@@ -310,19 +334,19 @@ namespace {
 // the address is looked up once per device (with that device current).
 pd_status static_scratch_ptr(void** out) {
   constexpr int kMaxDevices = 64;
-  static void* cached[kMaxDevices];
+  static std::atomic<void*> cached[kMaxDevices];  // two threads making the first call store the same address
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return record_cuda_error(e);
   if (dev < 0 || dev >= kMaxDevices) return PD_ERR_UNSUPPORTED;
-  if (!cached[dev]) {
-    void* ptr = nullptr;
+  void* ptr = cached[dev].load(std::memory_order_acquire);
+  if (!ptr) {
     e = cudaGetSymbolAddress(&ptr, g_layer_scratch);
     if (e != cudaSuccess) return record_cuda_error(e);
     if (!ptr) return PD_ERR_CUDA;
-    cached[dev] = ptr;
+    cached[dev].store(ptr, std::memory_order_release);
   }
-  *out = cached[dev];
+  *out = ptr;
   return PD_OK;
 }
 
@@ -335,9 +359,10 @@ extern "C" pd_status pd_encoder_layer_fwd_static(const pd_encoder_layer_desc* de
                                                  const pd_encoder_layer_weights* w, const void* x, void* y,
                                                  cudaStream_t stream) {
   using namespace pd;
-  if (!desc) return PD_ERR_NULL_POINTER;
-  if (!valid_desc(desc)) return PD_ERR_BAD_SHAPE;
-  if (!supported_desc(desc)) return PD_ERR_UNSUPPORTED;
+  // the same checks in the same order as pd_encoder_layer_fwd, so that an argument with several faults is
+  // reported alike by both; the size check comes where that call checks its workspace
+  if (pd_status st = check_layer_args(desc, w, x, y); st != PD_OK) return st;
+  if (desc->batch == 0) return PD_OK;
   if (plan(desc).total > PD_STATIC_SCRATCH_BYTES) return PD_ERR_WORKSPACE_TOO_SMALL;
   void* scratch = nullptr;
   pd_status st = static_scratch_ptr(&scratch);

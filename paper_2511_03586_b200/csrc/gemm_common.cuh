@@ -136,6 +136,9 @@ __device__ __forceinline__ void epilogue_warp(const KernelParams& p, const CUten
   const int my_steps = ((NCHUNK - group + 1) / 2) * STEPS;
   auto col_of = [&](int i) { return ((i / STEPS) * 2 + group) * CW + (i % STEPS) * 32; };
   int local = 0;
+  // A TMA store clips at the row's end only in whole 16-byte units.  When N elements are not a whole number of
+  // them, the chunk that holds the end of the row is written with plain stores instead.
+  const bool ragged_n = ((int64_t)p.N * (C_F32 ? 4 : 2)) % 16 != 0;
   if (lane == 0) prefetch_tensormap(tmap_c);
   for (int tile = first_tile; tile < p.num_tiles; tile += tile_stride, ++local) {
     const int nt = tile % p.tiles_n;
@@ -210,6 +213,20 @@ __device__ __forceinline__ void epilogue_warp(const KernelParams& p, const CUten
       float v[32];
 #pragma unroll
       for (int j = 0; j < 16; ++j) unpack_f32x2(v2[j], v[2 * j], v[2 * j + 1]);
+      if (ragged_n && n0 - step * 32 + CW > p.N) {
+        if (row_ok) {
+          const int64_t off = (int64_t)bo * p.strideC_outer + (int64_t)bi * p.strideC_inner + (int64_t)m * p.ldc + n0;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            if (n0 + j < p.N) {
+              if constexpr (C_F32) static_cast<float*>(p.C)[off + j] = v[j];
+              else static_cast<__nv_bfloat16*>(p.C)[off + j] = __float2bfloat16_rn(v[j]);
+            }
+          }
+        }
+        cur = nxt;
+        continue;
+      }
       if (step == 0) {
         // the previous store of this warp must have finished reading the buffer
         if (lane == 0) tma_store_wait_read<0>();

@@ -441,16 +441,17 @@ pd_status launch_ln_variant(const GemmProblem& g, const float* gamma, const floa
   cfg.numAttrs = 2;
   // Row blocks are dealt statically to the clusters, so launch only as many clusters as can be resident at once
   // (a cluster has to fit inside one GPC, which can leave a few SMs without one).
-  static int resident[kMaxCluster + 1];  // per cluster size, 0 = not queried yet
-  if (resident[ln.cluster] == 0) {
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) {
+  static std::atomic<int> resident[kMaxDevicesPerProcess][kMaxCluster + 1];  // per device and cluster size, 0 = not queried yet
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevicesPerProcess) return PD_ERR_UNSUPPORTED;
+  int clusters = resident[dev][ln.cluster].load(std::memory_order_relaxed);
+  if (clusters == 0) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg) != cudaSuccess || clusters < 1) {
       (void)cudaGetLastError();
-      n = 1;
+      clusters = 1;
     }
-    resident[ln.cluster] = n;
+    resident[dev][ln.cluster].store(clusters, std::memory_order_relaxed);
   }
-  int clusters = resident[ln.cluster];
   if (clusters > sm_count() / ln.cluster) clusters = sm_count() / ln.cluster;
   if (clusters > p.tiles_m) clusters = p.tiles_m;
   if (clusters < 1) clusters = 1;

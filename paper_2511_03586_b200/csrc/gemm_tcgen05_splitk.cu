@@ -351,6 +351,10 @@ pd_status launch_split_variant(const GemmProblem& g, cudaStream_t s) {
 int gemm_split_k_factor(const GemmProblem& g) {
   if (g.batch_inner != 1 || g.batch_outer != 1) return 0;
   if (g.B2 != nullptr && (g.b_is_nk || g.c_dtype != PD_BF16)) return 0;
+  // The epilogue of the split kernel stores, and reads bias and residual, eight whole columns at a time: a row
+  // whose length is not a multiple of eight is left to the kernels whose TMA stores clip the edge.
+  if (g.N % 8 != 0 || g.ldc % (g.c_dtype == PD_F32 ? 4 : 8) != 0 || (g.residual != nullptr && g.ldr % 8 != 0)) return 0;
+  if (g.bias != nullptr && !aligned16(g.bias)) return 0;
   const int64_t oc = g.B2 != nullptr ? 128 : 256;
   const int64_t tiles = ((g.M + BM - 1) / BM) * ((g.N + oc - 1) / oc);
   const int64_t num_kb = (g.K + BK - 1) / BK;

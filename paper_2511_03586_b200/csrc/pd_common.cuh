@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "pd.h"
 
 namespace pd {
@@ -27,7 +29,7 @@ int* device_status_ptr();
 // to the device's context, and one process may drive several devices).  `done` is the caller's per-kernel record.
 constexpr int kMaxDevicesPerProcess = 64;
 struct PerDeviceFlag {
-  bool set[kMaxDevicesPerProcess] = {};
+  std::atomic<bool> set[kMaxDevicesPerProcess] = {};  // concurrent first launches both set the attribute: harmless
 };
 template <typename Kernel>
 inline pd_status allow_dynamic_smem(Kernel kernel, int bytes, PerDeviceFlag& done) {
@@ -35,10 +37,10 @@ inline pd_status allow_dynamic_smem(Kernel kernel, int bytes, PerDeviceFlag& don
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return record_cuda_error(e);
   if (dev < 0 || dev >= kMaxDevicesPerProcess) return PD_ERR_UNSUPPORTED;
-  if (!done.set[dev]) {
+  if (!done.set[dev].load(std::memory_order_acquire)) {
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
     if (e != cudaSuccess) return record_cuda_error(e);
-    done.set[dev] = true;
+    done.set[dev].store(true, std::memory_order_release);
   }
   return PD_OK;
 }

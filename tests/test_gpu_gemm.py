@@ -170,6 +170,40 @@ def test_configured_shape_sampled_rows(api):
     assert torch.equal(c, c32.to(torch.bfloat16))
 
 
+# Row lengths that are not a multiple of eight elements: C sits in a wider matrix (ldc a legal multiple), and every
+# column from N on must keep its fill value.  K >= 2048 with few output tiles is the territory of the split-K
+# kernel, whose epilogue stores eight columns at a time: such shapes must be routed to the kernels that clip.
+@pytest.mark.parametrize("c_dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("b_is_nk", [False, True])
+@pytest.mark.parametrize("shape", [(128, 36, 2048), (128, 100, 2048), (200, 250, 4096), (130, 100, 72), (260, 257, 136),
+                                   (64, 4, 64), (300, 1001, 264), (130, 100, 100), (64, 72, 2051), (40, 33, 7)])
+def test_row_lengths_off_the_vector_width(api, shape, b_is_nk, c_dtype):
+    M, N, K = shape
+    p = inputs.gemm_integer_inputs(M, N, K, seed=M + N + K, b_is_nk=b_is_nk)
+    ref = _oracle(p, b_is_nk)[0]
+    if c_dtype == torch.bfloat16:
+        ref = inputs.bf16_bits_to_f32(inputs.f32_to_bf16_bits(ref.astype(np.float32))).astype(np.float64)
+    unit = 4 if c_dtype == torch.float32 else 8
+    # operands in wider matrices whose padding columns hold a large value: nothing beyond K or N may be read as data
+    lda = (K + 7) // 8 * 8
+    A = torch.full((M, lda), 3.0e4, dtype=torch.bfloat16, device="cuda")
+    A[:, :K] = dev_bf16(p["a_bits"][0])
+    b_rows, b_cols = (N, K) if b_is_nk else (K, N)
+    ldb = (b_cols + 7) // 8 * 8
+    B = torch.full((b_rows, ldb), 3.0e4, dtype=torch.bfloat16, device="cuda")
+    B[:, :b_cols] = dev_bf16(p["b_bits"][0])
+    for ldc in ((N + unit - 1) // unit * unit, (N + unit - 1) // unit * unit + 3 * unit):
+        c = Guarded((M, ldc), c_dtype)
+        c.t.fill_(-7.0)
+        st = api.pd_gemm_bf16_raw(A.data_ptr(), B.data_ptr(), c.t.data_ptr(), M, N, K, lda, ldb, ldc, b_is_nk,
+                                  api.PD_F32 if c_dtype == torch.float32 else api.PD_BF16, 1, 0, 0, 0)
+        assert st == 0
+        torch.cuda.synchronize()
+        c.check()
+        assert np.array_equal(host(c.t[:, :N]), ref)
+        assert bool((c.t[:, N:] == -7.0).all()), "columns outside C were written"
+
+
 def test_strided_operands_and_errors(api):
     # operands embedded in wider matrices (ld > row length), addressed through the raw entry point
     M, N, K = 96, 80, 72

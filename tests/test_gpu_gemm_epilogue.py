@@ -142,6 +142,21 @@ def test_split_k_over_a_cluster_matches_the_unsplit_kernel(api, shape):
     assert max_rel_floored(outs[0], outs[1]) < 1e-5
 
 
+def test_layer_ffn_up_launch_sampled_rows(api):
+    # the layer's FFN-up launch at full size (16384 x 4096 x 1024, bias + GELU, bf16 out), under every tile mode of
+    # the fixture (the layer itself takes the CTA-pair kernel): sampled rows from every part of the tile walk
+    M, K, N = 16384, 1024, 4096
+    p = inputs.gemm_layernorm_inputs(M, N, K, seed=11)
+    c = api.pd_gemm_bias_act(dev_bf16(p["a_bits"]), dev_bf16(p["b_bits"]), dev_f32(p["bias"]), None, act=api.ACT_GELU)
+    pick = np.unique(np.concatenate([[0, 127, 128, 255, 256, M - 257, M - 256, M - 129, M - 128, M - 1],
+                                     np.random.default_rng(11).integers(0, M, 60)]))
+    ref = oracle.bias_gelu_residual(oracle.gemm(p["a"][pick], p["b"]), p["bias"], None)
+    err = max_rel_floored(host(c[torch.from_numpy(pick).cuda()]), ref)
+    assert err < TOL
+    assert err < TOL_ONE_ROUNDING
+    assert bool(torch.isfinite(c.float()).all())
+
+
 def test_argument_errors(api):
     from paper_2511_03586_b200.api import PdError
     a = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")

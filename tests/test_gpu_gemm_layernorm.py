@@ -62,6 +62,26 @@ def test_against_oracle(api, shape):
     assert err < TOL_ONE_ROUNDING
 
 
+# The layer's two LayerNorm launches at full size: output projection (K = 1024) and FFN down (K = 4096), 16384 rows
+# of 1024 columns.  The oracle is run on sampled rows from every part of the walk over the row blocks (first and
+# last block, block edges, a random spread): a row's result depends on that row of A and of the residual only.
+@pytest.mark.parametrize("K", [1024, 4096])
+def test_layer_shapes_sampled_rows(api, K):
+    M, N = 16384, 1024
+    p = inputs.gemm_layernorm_inputs(M, N, K, seed=K)
+    y = api.pd_gemm_bias_residual_layernorm(dev_bf16(p["a_bits"]), dev_bf16(p["b_bits"]), dev_f32(p["bias"]),
+                                            dev_bf16(p["residual_bits"]), dev_f32(p["gamma"]), dev_f32(p["beta"]),
+                                            p["eps"])
+    pick = np.unique(np.concatenate([[0, 31, 32, 127, 128, M - 129, M - 128, M - 33, M - 1],
+                                     np.random.default_rng(K).integers(0, M, 60)]))
+    s = oracle.gemm(p["a"][pick], p["b"]) + p["bias"].astype(np.float64) + p["residual"][pick].astype(np.float64)
+    ref = oracle.layernorm(s, p["gamma"], p["beta"], np.float32(p["eps"]))
+    err = max_rel_floored(host(y[torch.from_numpy(pick).cuda()]), ref)
+    assert err < TOL
+    assert err < TOL_ONE_ROUNDING
+    assert bool(torch.isfinite(y.float()).all())
+
+
 @pytest.mark.parametrize("use_bias,use_residual", [(False, False), (True, False), (False, True)])
 def test_optional_operands(api, use_bias, use_residual):
     p = inputs.gemm_layernorm_inputs(333, 768, 264, seed=5)

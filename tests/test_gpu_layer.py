@@ -116,7 +116,7 @@ def test_attention_peaked_rows_and_errors(api):
 # (batch, seq, heads, ffn): seq <= 512 takes the fused attention kernel, 640 the unfused path
 @pytest.mark.parametrize("dims", [(2, 64, 2, 256), (3, 136, 1, 72), (1, 512, 4, 1024), (5, 8, 3, 8), (2, 100, 2, 64),
                                   (1, 640, 1, 128)])
-@pytest.mark.parametrize("w_sigma", [0.02, 0.05])
+@pytest.mark.parametrize("w_sigma", [0.02, 0.05, 0.08])
 def test_small_layers(api, dims, w_sigma):
     batch, seq, heads, ffn = dims
     shape = inputs.EncoderLayerShape(batch=batch, seq=seq, hidden=64 * heads, heads=heads, ffn=ffn)
@@ -149,16 +149,66 @@ def test_bert_large_shape_sampled_sequences(api):
     y2 = api.pd_encoder_layer_fwd(params, x, batch=shape.batch, seq=shape.seq, heads=shape.heads, workspace=ws)
     assert torch.equal(y, y2)                           # deterministic
     assert bool(torch.isfinite(y.float()).all())
-    # sequences are independent, so the oracle is run on one of them (about 7 G multiply-adds)
-    b = 17
-    rows = slice(b * shape.seq, (b + 1) * shape.seq)
-    ref = _oracle_layer(p, shape, rows=rows, batch=1)
-    assert max_rel_floored(host(y[rows]), ref) < TOL
+    # sequences are independent, so the oracle is run on three of them (about 7 G multiply-adds each): the first
+    # and the last, which sit at the two ends of the attention kernel's and the FFN-down launch's reversed walks,
+    # and one from the middle
+    for b in (0, 17, shape.batch - 1):
+        rows = slice(b * shape.seq, (b + 1) * shape.seq)
+        ref = _oracle_layer(p, shape, rows=rows, batch=1)
+        assert max_rel_floored(host(y[rows]), ref) < TOL, f"sequence {b}"
     # property that holds at any size: every output row, un-affined, has zero mean and unit variance
     g2, b2 = dev_f32(p["ln2_gamma"]), dev_f32(p["ln2_beta"])
     z = (y.float() - b2) / g2
     assert float(z.mean(dim=1).abs().max()) < 0.05
     assert float((z.var(dim=1, unbiased=False) - 1).abs().max()) < 0.05
+
+
+def test_bert_large_shape_every_launch_on_sampled_rows(api):
+    """Each launch of the full-size layer on its own: the oracle recomputes a stage's output for sampled rows from
+    the stage's INPUT as the GPU produced it (read back from the workspace), so a fault in one launch cannot hide
+    behind the tolerance of the stages after it, and every launch is checked in the configuration the benchmark
+    times (CTA-pair tiles, LayerNorm epilogues, FFN-down and attention walking their rows last first)."""
+    shape = inputs.EncoderLayerShape()
+    T, H, F, S = shape.tokens, shape.hidden, shape.ffn, shape.seq
+    p = inputs.encoder_layer_inputs(shape, seed=1)
+    params = _device_params(api, p)
+    x = dev_bf16(p["x_bits"])
+    dims = (shape.batch, S, H, shape.heads, F)
+    ws = torch.empty(api.pd_encoder_layer_workspace_bytes(*dims), dtype=torch.uint8, device="cuda")
+    y = api.pd_encoder_layer_fwd(params, x, batch=shape.batch, seq=S, heads=shape.heads, workspace=ws)
+    torch.cuda.synchronize()
+    lay = api.pd_encoder_layer_workspace_layout(*dims)
+
+    def buf(name, cols):
+        off, size = lay[name]
+        assert size >= T * cols * 2
+        return ws[off:off + T * cols * 2].view(torch.bfloat16).view(T, cols)
+
+    qkv, ctx, h1, mid = buf("qkv", 3 * H), buf("ctx", H), buf("h1", H), buf("mid", F)
+    w = {m: inputs.bf16_bits_to_f32(p[m + "_bits"]) for m in _MATS}
+    pick = np.unique(np.concatenate([[0, 127, 128, 255, 256, T - 257, T - 256, T - 129, T - 128, T - 1],
+                                     np.random.default_rng(3).integers(0, T, 50)]))
+    idx = torch.from_numpy(pick).cuda()
+    one_rounding = 2.0 ** -8
+    # QKV projection
+    ref = oracle.gemm(host(x[idx]), w["w_qkv"]) + p["b_qkv"].astype(np.float64)
+    assert max_rel_floored(host(qkv[idx]), ref) < one_rounding
+    # attention, whole sequences (first, last, one in the middle), from the GPU's own qkv
+    for b in (0, 13, shape.batch - 1):
+        rows = slice(b * S, (b + 1) * S)
+        ref = oracle.attention(host(qkv[rows]), 1, S, shape.heads, 64)
+        assert max_rel_floored(host(ctx[rows]), ref) < TOL, f"attention, sequence {b}"
+    # output projection + residual + LayerNorm
+    s = oracle.gemm(host(ctx[idx]), w["w_o"]) + p["b_o"].astype(np.float64) + host(x[idx])
+    ref = oracle.layernorm(s, p["ln1_gamma"], p["ln1_beta"], np.float32(shape.ln_eps))
+    assert max_rel_floored(host(h1[idx]), ref) < one_rounding
+    # FFN up + GELU
+    ref = oracle.bias_gelu_residual(oracle.gemm(host(h1[idx]), w["w_ffn1"]), p["b_ffn1"], None)
+    assert max_rel_floored(host(mid[idx]), ref) < one_rounding
+    # FFN down + residual + LayerNorm
+    s = oracle.gemm(host(mid[idx]), w["w_ffn2"]) + p["b_ffn2"].astype(np.float64) + host(h1[idx])
+    ref = oracle.layernorm(s, p["ln2_gamma"], p["ln2_beta"], np.float32(shape.ln_eps))
+    assert max_rel_floored(host(y[idx]), ref) < one_rounding
 
 
 def test_stack_of_layers_against_oracle(api):

@@ -77,6 +77,30 @@ def test_layernorm_shapes(api, cols):
             assert max_rel_floored(host(y.t), ref) < TOL
 
 
+# Many rows (several waves of CTAs, a ragged last one) for each kernel family: a warp per row, and CTAs of 64, 128
+# and 256 threads per row, with ragged row lengths within them.
+@pytest.mark.parametrize("dims", [(5000, 512), (9001, 1024), (4099, 1000), (3001, 2048), (2100, 1540), (1501, 4096),
+                                  (1300, 2052), (777, 8192), (700, 4100)])
+def test_many_rows(api, dims):
+    rows, cols = dims
+    p = inputs.layernorm_inputs(rows, cols, seed=cols)
+    x, g, b = dev_f32(p["x"]), dev_f32(p["gamma"]), dev_f32(p["beta"])
+    y = Guarded((rows, cols), torch.float32)
+    api.pd_layernorm(x, g, b, p["eps"], y.t)
+    torch.cuda.synchronize()
+    y.check()
+    assert max_rel_floored(host(y.t), oracle.layernorm(p["x"], p["gamma"], p["beta"], np.float32(p["eps"]))) < TOL
+    z = Guarded((rows, cols), torch.float32)
+    api.pd_rmsnorm(x, g, p["eps"], z.t)
+    torch.cuda.synchronize()
+    z.check()
+    assert max_rel_floored(host(z.t), oracle.rmsnorm(p["x"], p["gamma"], np.float32(p["eps"]))) < TOL
+    # in place, and repeatable
+    x2 = x.clone()
+    api.pd_layernorm(x2, g, b, p["eps"], x2)
+    assert torch.equal(x2, y.t)
+
+
 def test_layernorm_configured_and_paper_shapes(api):
     for rows, cols in ((4096, 1024), (16384, 1024), (4096, 4096)):
         p = inputs.layernorm_inputs(rows, cols, seed=0)

@@ -163,3 +163,26 @@ def test_attention_and_layer(lib):
     assert lib.pd_encoder_layer_workspace_bytes(ctypes.byref(big)) > lib.pd_encoder_layer_static_scratch_bytes()
     assert lib.pd_encoder_layer_fwd_static(ctypes.byref(big), ctypes.byref(w), P, P, None) == WS_SMALL
     assert lib.pd_encoder_layer_fwd_static(None, ctypes.byref(w), P, P, None) == NULLP
+    # faults are reported in the same order as by pd_encoder_layer_fwd: a null or misaligned x before the size
+    assert lib.pd_encoder_layer_fwd_static(ctypes.byref(big), ctypes.byref(w), None, P, None) == NULLP
+    assert lib.pd_encoder_layer_fwd_static(ctypes.byref(big), ctypes.byref(w), P + 8, P, None) == ALIGN
+    assert lib.pd_encoder_layer_fwd_static(ctypes.byref(big), ctypes.byref(missing), P, P, None) == NULLP
+    # more tokens than an int can index
+    huge = Desc(1 << 23, 512, 256, 4, 512, 1e-5)
+    assert lib.pd_encoder_layer_fwd(ctypes.byref(huge), ctypes.byref(w), P, P, P, need, None) == SHAPE
+    assert lib.pd_encoder_layer_workspace_bytes(ctypes.byref(huge)) == 0
+
+    # where the intermediates sit inside the workspace: consecutive, 256-byte aligned, adding up to the total
+    n = 7
+    off, size = (ctypes.c_size_t * n)(), (ctypes.c_size_t * n)()
+    lib.pd_encoder_layer_workspace_layout.argtypes = [ctypes.POINTER(Desc), ctypes.POINTER(ctypes.c_size_t),
+                                                      ctypes.POINTER(ctypes.c_size_t)]
+    assert lib.pd_encoder_layer_workspace_layout(ctypes.byref(good), off, size) == OK
+    assert off[0] == 0 and all(off[i] + size[i] == off[i + 1] for i in range(n - 1)) and off[n - 1] + size[n - 1] == need
+    assert all(o % 256 == 0 for o in off)
+    T, H, F = 2 * 128, 256, 512
+    assert size[0] == T * 3 * H * 2 and size[3] == T * H * 2 and size[5] == T * H * 2 and size[6] == T * F * 2
+    assert size[1] == 0 and size[2] == 0          # fused attention keeps scores and probabilities on the SM
+    assert lib.pd_encoder_layer_workspace_layout(None, off, size) == NULLP
+    assert lib.pd_encoder_layer_workspace_layout(ctypes.byref(good), None, size) == NULLP
+    assert lib.pd_encoder_layer_workspace_layout(ctypes.byref(Desc(2, 0, 256, 4, 512, 1e-5)), off, size) == SHAPE
