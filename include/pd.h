@@ -75,6 +75,22 @@ int pd_last_cuda_error(void);
 pd_status pd_get_device_status(int* code);
 pd_status pd_clear_device_status(void);
 
+/* Test aids for the bounded waits (the analogue of the run and compile
+ * time-outs of the paper's search loop, Sections 4.2.3 "Performance on x86" and
+ * 4.3 "Search with PerfLLM": a candidate that does not finish is cut off and
+ * reported, it does not take the system down).
+ * pd_debug_set_wait_limit_ns: the time after which a wait inside the single-CTA
+ * contraction kernel (pd_set_gemm_tile_mode(1)) gives up, 1 us to 10 s (else
+ * PD_ERR_BAD_SHAPE); default 2 s.  pd_debug_withhold_loads(1): that kernel's
+ * producer thread issues no load, so the thread that feeds the tensor core
+ * waits for its first operand stage in vain, gives up after the limit, records
+ * code 102 in the device status word, and every role of the kernel drains and
+ * returns (nothing faults, traps or stays behind; the output is not written).
+ * pd_debug_withhold_loads(0) restores normal operation.  Both settings are
+ * process-wide and apply to launches enqueued after the call. */
+pd_status pd_debug_set_wait_limit_ns(uint64_t limit_ns);
+pd_status pd_debug_withhold_loads(int on);
+
 /* Row-wise softmax over the last dimension (operator "softmax" of the paper's
  * operator table; reduction, broadcast and element-wise features):
  *   y[i,j] = exp(x[i,j] - m_i) / sum_j exp(x[i,j] - m_i),  m_i = max_j x[i,j].

@@ -57,6 +57,8 @@ def _load() -> ctypes.CDLL:
     lib.pd_last_cuda_error.argtypes = []; lib.pd_last_cuda_error.restype = ctypes.c_int
     lib.pd_get_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]; lib.pd_get_device_status.restype = st
     lib.pd_clear_device_status.argtypes = []; lib.pd_clear_device_status.restype = st
+    lib.pd_debug_set_wait_limit_ns.argtypes = [ctypes.c_uint64]; lib.pd_debug_set_wait_limit_ns.restype = st
+    lib.pd_debug_withhold_loads.argtypes = [ctypes.c_int]; lib.pd_debug_withhold_loads.restype = st
     lib.pd_softmax.argtypes = [vp, vp, i64, i64, vp]; lib.pd_softmax.restype = st
     lib.pd_layernorm.argtypes = [vp, vp, vp, vp, i64, i64, ctypes.c_float, vp]; lib.pd_layernorm.restype = st
     lib.pd_rmsnorm.argtypes = [vp, vp, vp, i64, i64, ctypes.c_float, vp]; lib.pd_rmsnorm.restype = st
@@ -415,3 +417,13 @@ def pd_get_device_status() -> int:
 
 def pd_clear_device_status() -> None:
     _check(_lib.pd_clear_device_status(), "pd_clear_device_status")
+
+
+def pd_debug_set_wait_limit_ns(limit_ns: int) -> None:
+    """Time after which a wait inside the single-CTA contraction kernel gives up (default 2 s)."""
+    _check(_lib.pd_debug_set_wait_limit_ns(int(limit_ns)), "pd_debug_set_wait_limit_ns")
+
+
+def pd_debug_withhold_loads(on: bool) -> None:
+    """Test switch: the single-CTA contraction kernel's producer issues no load, so a bounded wait runs out."""
+    _check(_lib.pd_debug_withhold_loads(int(bool(on))), "pd_debug_withhold_loads")

@@ -14,6 +14,13 @@ __device__ int g_device_status;
 
 }  // namespace
 
+namespace {
+std::atomic<uint64_t> g_wait_limit_ns{2000000000ull};
+std::atomic<int> g_withhold_loads{0};
+}  // namespace
+uint64_t debug_wait_limit_ns() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
+int debug_withhold_loads() { return g_withhold_loads.load(std::memory_order_relaxed); }
+
 pd_status record_cuda_error(cudaError_t e) {
   if (e == cudaSuccess) return PD_OK;
   tl_last_cuda_error = (int)e;
@@ -98,4 +105,16 @@ extern "C" pd_status pd_clear_device_status(void) {
   cudaError_t e = cudaDeviceSynchronize();
   if (e == cudaSuccess) e = cudaMemset(p, 0, sizeof(int));
   return pd::record_cuda_error(e);
+}
+
+extern "C" pd_status pd_debug_set_wait_limit_ns(uint64_t limit_ns) {
+  if (limit_ns < 1000ull || limit_ns > 10000000000ull) return PD_ERR_BAD_SHAPE;
+  pd::g_wait_limit_ns.store(limit_ns, std::memory_order_relaxed);
+  return PD_OK;
+}
+
+extern "C" pd_status pd_debug_withhold_loads(int on) {
+  if (on < 0 || on > 1) return PD_ERR_BAD_SHAPE;
+  pd::g_withhold_loads.store(on, std::memory_order_relaxed);
+  return PD_OK;
 }

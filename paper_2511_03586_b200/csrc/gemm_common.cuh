@@ -29,7 +29,15 @@ struct KernelParams {
   int tiles_m, tiles_n, batch_inner, num_tiles;  // num_tiles = batch_outer * batch_inner * tiles_m * tiles_n
   float alpha;
   int c_is_f32, act;  // act: 0 nothing, 1 erf-form GELU, 2 ReLU
+  // Single-CTA kernel only (zero elsewhere): the time after which its waits give up (0: the default of 2 s), and
+  // the test switch that makes its producer skip every load, so that the wait for the first stage runs out.
+  unsigned long long wait_limit_ns;
+  int withhold_loads;
 };
+
+__device__ __forceinline__ uint64_t wait_limit(const KernelParams& p) {
+  return p.wait_limit_ns != 0 ? (uint64_t)p.wait_limit_ns : 2000000000ull;
+}
 
 // Codes left in the device status word by an expired wait.
 enum : int { kTimeoutProducer = 101, kTimeoutMmaFull = 102, kTimeoutMmaAcc = 103, kTimeoutEpilogue = 104 };
@@ -154,7 +162,7 @@ __device__ __forceinline__ void epilogue_warp(const KernelParams& p, const CUten
     ResidualRegs cur, nxt;
     if (my_steps > 0 && n_tile + col_of(0) < p.N)
       cur.load(p, m, n_tile + col_of(0), row_ok);  // independent of the accumulator: issued before the wait
-    if (!mbar_wait(acc_full_bar0 + 8u * acc, acc_ph, abort_flag, p.status, kTimeoutEpilogue)) break;
+    if (!mbar_wait(acc_full_bar0 + 8u * acc, acc_ph, abort_flag, p.status, kTimeoutEpilogue, wait_limit(p))) break;
     tcgen05_fence_after_sync();
     const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
 #pragma unroll 1
@@ -291,7 +299,7 @@ __device__ __forceinline__ void epilogue_warp_gated(const KernelParams& p, const
     const int acc = local & 1;
     const uint32_t acc_ph = (local >> 1) & 1u;
     const int m_warp = mt * BM + quarter * 32;
-    if (!mbar_wait(acc_full_bar0 + 8u * acc, acc_ph, abort_flag, p.status, kTimeoutEpilogue)) break;
+    if (!mbar_wait(acc_full_bar0 + 8u * acc, acc_ph, abort_flag, p.status, kTimeoutEpilogue, wait_limit(p))) break;
     tcgen05_fence_after_sync();
     const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
 #pragma unroll 1

@@ -107,7 +107,8 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       if (GATED) prefetch_tensormap(&tmap_b2);
       uint32_t it = 0;  // k-blocks issued so far, over all tiles
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x) {
+      // (test switch: with withhold_loads set the producer issues nothing, and the wait for the first stage runs out)
+      for (int tile = blockIdx.x; tile < p.num_tiles && ok && !p.withhold_loads; tile += gridDim.x) {
         const int nt = tile % p.tiles_n;
         const int mt = (tile / p.tiles_n) % p.tiles_m;
         const int b = tile / (p.tiles_n * p.tiles_m);
@@ -115,7 +116,7 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer, wait_limit(p))) { ok = false; break; }
           const uint32_t sa = smem_base + s * C::kStage, sb = sa + C::kStageA;
           mbar_arrive_expect_tx(full_bar(s), C::kStage);
           tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, bi, bo);
@@ -154,13 +155,13 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local) {
         const int acc = local & 1;
         const uint32_t acc_ph = (local >> 1) & 1u;
-        if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc)) { ok = false; break; }
+        if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc, wait_limit(p))) { ok = false; break; }
         tcgen05_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
+          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull, wait_limit(p))) { ok = false; break; }
           tcgen05_fence_after_sync();
           const uint32_t sa = smem_base + s * C::kStage, sb = sa + C::kStageA;
 #pragma unroll
@@ -235,6 +236,8 @@ pd_status launch_variant(const GemmProblem& g, cudaStream_t s) {
   if (tiles > 0x7fffffff) return PD_ERR_BAD_SHAPE;
   p.num_tiles = (int)tiles;
   p.alpha = g.alpha; p.c_is_f32 = g.c_dtype == PD_F32; p.act = g.act;
+  p.wait_limit_ns = debug_wait_limit_ns();
+  p.withhold_loads = debug_withhold_loads();
 
   auto kernel = gemm_bf16_tcgen05_kernel<BN, B_NK, C_F32, GATED>;
   static PerDeviceFlag smem_allowed;  // one per kernel (template instantiation)

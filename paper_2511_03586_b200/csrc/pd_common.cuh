@@ -24,6 +24,11 @@ pd_status require_sm100();
 int sm_count();
 // Device address of the status word the bounded waits report to (nullptr on failure).
 int* device_status_ptr();
+// Test aids behind pd_debug_set_wait_limit_ns / pd_debug_withhold_loads: the time after which a wait inside the
+// single-CTA contraction kernel gives up (default 2 s), and whether that kernel's producer skips its loads, so
+// that the wait for them runs out.
+uint64_t debug_wait_limit_ns();
+int debug_withhold_loads();
 
 // Raises the dynamic shared-memory limit of `kernel` on the current device, once per device (the attribute belongs
 // to the device's context, and one process may drive several devices).  `done` is the caller's per-kernel record.
