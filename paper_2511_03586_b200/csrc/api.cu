@@ -1,5 +1,8 @@
 // Status handling, device checks and the device status word of the pd library.
 #include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
 
 #include "pd_common.cuh"
 
@@ -20,6 +23,23 @@ std::atomic<int> g_withhold_loads{0};
 }  // namespace
 uint64_t debug_wait_limit_ns() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
 int debug_withhold_loads() { return g_withhold_loads.load(std::memory_order_relaxed); }
+
+bool log_enabled() {
+  static const bool on = [] {
+    const char* v = std::getenv("PD_LOG");
+    return v != nullptr && v[0] != '\0' && v[0] != '0';
+  }();
+  return on;
+}
+void logf(const char* fmt, ...) {
+  if (!log_enabled()) return;
+  va_list ap;
+  va_start(ap, fmt);
+  std::fputs("pd: ", stderr);
+  std::vfprintf(stderr, fmt, ap);
+  std::fputc('\n', stderr);
+  va_end(ap);
+}
 
 pd_status record_cuda_error(cudaError_t e) {
   if (e == cudaSuccess) return PD_OK;

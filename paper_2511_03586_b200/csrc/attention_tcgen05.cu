@@ -620,6 +620,8 @@ pd_status launch_fused_attention(const __nv_bfloat16* qkv, __nv_bfloat16* ctx, i
   static PerDeviceFlag smem_allowed;  // one per kernel (template instantiation)
   if (pd_status st = allow_dynamic_smem(attention_fwd_tcgen05_kernel, kSmemBytes, smem_allowed); st != PD_OK) return st;
   const int grid = p.num_units < sm_count() ? p.num_units : sm_count();
+  logf("attention batch %lld seq %lld heads %lld: fused kernel, %d work units on %d CTAs", (long long)batch, (long long)seq,
+       (long long)heads, p.num_units, grid);
   launch_pdl(attention_fwd_tcgen05_kernel, dim3(grid), dim3(kThreads), kSmemBytes, s, tq, tk, tv, to, p);
   return check_launch();
 }

@@ -11,6 +11,8 @@
 // LayerNorm GEMMs write their fp32 sum to a scratch tensor and the LayerNorm row kernel follows.
 #include <atomic>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "pd_common.cuh"
 
 namespace pd {
@@ -95,6 +97,8 @@ namespace {
 constexpr int kStages = 7;
 const char* const kStageNames[kStages] = {"qkv_gemm", "attention", "out_proj_gemm", "layernorm1",
                                           "ffn_up_gemm", "ffn_down_gemm", "layernorm2"};
+const char* const kStageRangeNames[kStages] = {"pd.qkv_gemm", "pd.attention", "pd.out_proj_gemm", "pd.layernorm1",
+                                               "pd.ffn_up_gemm", "pd.ffn_down_gemm", "pd.layernorm2"};
 
 // Argument checks shared by every layer entry point: null pointers, then the shape, then alignment.
 pd_status check_layer_args(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* w, const void* x,
@@ -116,11 +120,23 @@ pd_status check_layer_args(const pd_encoder_layer_desc* desc, const pd_encoder_l
 // ev[i] is recorded before stage i and ev[kStages] after the last one.
 pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_weights* w, const void* x, void* y,
                     void* workspace, size_t workspace_bytes, cudaStream_t stream, cudaEvent_t* ev) {
+  // Every stage is bracketed by an NVTX range named after it (host side, around the enqueueing calls), so that a
+  // timeline tool shows the layer's structure; without a tool attached the calls do nothing.
   int stage = 0;
+  bool range_open = false;
   auto mark = [&]() {
+    if (range_open) nvtxRangePop();
+    range_open = stage < kStages;
+    if (range_open) nvtxRangePushA(kStageRangeNames[stage]);
     if (ev) cudaEventRecord(ev[stage], stream);
     ++stage;
   };
+  struct RangeGuard {  // closes the open range on every return path
+    bool& open;
+    ~RangeGuard() {
+      if (open) nvtxRangePop();
+    }
+  } guard{range_open};
   if (pd_status st0 = check_layer_args(desc, w, x, y); st0 != PD_OK) return st0;
   if (desc->batch == 0) return PD_OK;
   const Workspace ws = plan(desc);
@@ -131,6 +147,9 @@ pd_status run_layer(const pd_encoder_layer_desc* desc, const pd_encoder_layer_we
   if (st != PD_OK) return st;
 
   const int64_t B = desc->batch, S = desc->seq, H = desc->hidden, NH = desc->heads, F = desc->ffn, T = B * S;
+  logf("encoder layer batch %lld seq %lld hidden %lld heads %lld ffn %lld: attention %s, LayerNorms %s", (long long)B,
+       (long long)S, (long long)H, (long long)NH, (long long)F, use_fused_attention(desc) ? "fused" : "as three launches",
+       use_fused_layernorm(desc) ? "in the contractions' epilogues" : "as row kernels");
   uint8_t* base = static_cast<uint8_t*>(workspace);
   auto* qkv = reinterpret_cast<__nv_bfloat16*>(base + ws.qkv);
   auto* scores = reinterpret_cast<float*>(base + ws.scores);

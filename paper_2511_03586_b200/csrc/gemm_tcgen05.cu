@@ -268,7 +268,11 @@ void set_gemm_split_k_mode(int mode) { g_split_k_mode = mode; }
 pd_status launch_gemm(const GemmProblem& g, cudaStream_t s) {
   if (g_tile_mode == 0 && g_split_k_mode != 1) {
     const int split = gemm_split_k_factor(g);
-    if (split > 0 && (g.B2 == nullptr || (!g.bias && !g.residual && !g.act))) return launch_gemm_split_k(g, split, s);
+    if (split > 0 && (g.B2 == nullptr || (!g.bias && !g.residual && !g.act))) {
+      logf("gemm %lld x %lld x %lld%s: 128 x 256 tiles, K split over clusters of %d CTAs", (long long)g.M, (long long)g.N,
+           (long long)g.K, g.B2 ? " (gated)" : "", split);
+      return launch_gemm_split_k(g, split, s);
+    }
   }
   if (g.B2 != nullptr) {
     // gated form: 128 x 128 output tiles, or 128 x 64 when those fill the SMs' last wave better
@@ -277,9 +281,15 @@ pd_status launch_gemm(const GemmProblem& g, cudaStream_t s) {
     const int64_t tiles_m = (g.M + BM - 1) / BM, sms = sm_count();
     const int64_t t128 = tiles_m * ((g.N + 127) / 128), t64 = tiles_m * ((g.N + 63) / 64);
     const double c128 = (double)((t128 + sms - 1) / sms) * 256.0, c64 = (double)((t64 + sms - 1) / sms) * 128.0 / 0.66;
+    logf("gemm %lld x %lld x %lld (gated): 128 x %d output tiles, one CTA each", (long long)g.M, (long long)g.N,
+         (long long)g.K, c64 < c128 ? 64 : 128);
     return c64 < c128 ? launch_variant<128, false, false, true>(g, s) : launch_variant<256, false, false, true>(g, s);
   }
-  if (g_tile_mode == 2 || (g_tile_mode == 0 && gemm_pair_tiles_profitable(g))) return launch_gemm_pair(g, s);
+  if (g_tile_mode == 2 || (g_tile_mode == 0 && gemm_pair_tiles_profitable(g))) {
+    logf("gemm %lld x %lld x %lld batch %lld: 256 x 256 tiles on CTA pairs", (long long)g.M, (long long)g.N, (long long)g.K,
+         (long long)(g.batch_inner * g.batch_outer));
+    return launch_gemm_pair(g, s);
+  }
   // 128 x 256 tiles reuse operands best (the 128 x 128 main loop runs at about
   // two thirds of their rate); narrower tiles are used when N is small or when
   // they fill the last wave of SMs so much better that it pays.
@@ -293,6 +303,8 @@ pd_status launch_gemm(const GemmProblem& g, cudaStream_t s) {
   if (g.N <= 64) bn = 64;
   else if (g.N <= 128) bn = 128;
   else if (cost(128, 0.66) < cost(256, 1.0)) bn = 128;
+  logf("gemm %lld x %lld x %lld batch %lld: 128 x %d tiles, one CTA each", (long long)g.M, (long long)g.N, (long long)g.K,
+       (long long)(g.batch_inner * g.batch_outer), bn);
   if (bn == 256) return launch_bn<256>(g, s);
   if (bn == 128) return launch_bn<128>(g, s);
   return launch_bn<64>(g, s);

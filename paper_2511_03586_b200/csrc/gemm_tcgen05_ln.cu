@@ -456,6 +456,8 @@ pd_status launch_ln_variant(const GemmProblem& g, const float* gamma, const floa
   if (clusters > p.tiles_m) clusters = p.tiles_m;
   if (clusters < 1) clusters = 1;
   cfg.gridDim = dim3(clusters * ln.cluster);
+  logf("gemm + layernorm %lld x %lld x %lld: %d clusters of %d CTAs, rows %s", (long long)g.M, (long long)g.N, (long long)g.K,
+       clusters, ln.cluster, g.rows_descending ? "last first" : "first first");
   cudaLaunchKernelEx(&cfg, kernel, ta, tb, tc, p, ln);
   return check_launch();
 }

@@ -258,6 +258,11 @@ pd_status dispatch(const float* x, const float* g, const float* b, OutT* y, int6
                    cudaStream_t s) {
   const bool vec_ok = (cols % 4 == 0) && aligned16(x) && aligned16(g) && aligned16(b) &&
                       ((reinterpret_cast<uintptr_t>(y) & (sizeof(OutT) * 4 - 1)) == 0);
+  logf("%s %lld x %lld: %s", "layernorm", (long long)rows, (long long)cols,
+       !vec_ok ? "scalar three-pass path (unaligned or ragged rows)"
+       : cols <= 1024 ? "one warp per row, row in registers"
+       : cols <= 28672 ? "one CTA per row, row in registers"
+       : cols <= 262144 ? "one cluster per row, row in registers" : "one CTA per row, streaming passes");
   if (vec_ok && cols <= 1024) {
     const int c = (int)cols;
     if (c <= 128) launch_warp_rows<1>(x, g, b, y, rows, c, eps, s);

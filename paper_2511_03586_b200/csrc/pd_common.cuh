@@ -29,6 +29,10 @@ int* device_status_ptr();
 // that the wait for them runs out.
 uint64_t debug_wait_limit_ns();
 int debug_withhold_loads();
+// Variant-selection log: with PD_LOG=1 in the environment every launcher writes one line to stderr naming the
+// kernel variant it chose (read once per process; costs one branch otherwise).
+bool log_enabled();
+void logf(const char* fmt, ...) __attribute__((format(printf, 1, 2)));
 
 // Raises the dynamic shared-memory limit of `kernel` on the current device, once per device (the attribute belongs
 // to the device's context, and one process may drive several devices).  `done` is the caller's per-kernel record.

@@ -125,6 +125,9 @@ pd_status launch_rmsnorm(const float* x, const float* g, float* y, int64_t rows,
                          cudaStream_t s) {
   const bool vec_ok = (cols % 4 == 0) && aligned16(x) && aligned16(g) && aligned16(y);
   const int c = (int)cols;
+  logf("rmsnorm %lld x %lld: %s", (long long)rows, (long long)cols,
+       !vec_ok ? "scalar path (unaligned or ragged rows)" : cols <= 1024 ? "one warp per row, row in registers"
+       : cols <= 32768 ? "one CTA per row, row in registers" : cols <= 262144 ? "one cluster per row, row in registers" : "scalar path");
   if (vec_ok && cols <= 1024) {
     if (c <= 128) launch_warp_rows<1>(x, g, y, rows, c, eps, s);
     else if (c <= 256) launch_warp_rows<2>(x, g, y, rows, c, eps, s);

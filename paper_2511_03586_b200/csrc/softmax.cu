@@ -186,6 +186,11 @@ void launch_cta_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStream
 template <typename OutT>
 pd_status dispatch(const float* x, OutT* y, int64_t rows, int64_t cols, cudaStream_t s) {
   const bool vec_ok = (cols % 4 == 0) && aligned16(x) && ((reinterpret_cast<uintptr_t>(y) & (sizeof(OutT) * 4 - 1)) == 0);
+  logf("%s %lld x %lld: %s", "softmax", (long long)rows, (long long)cols,
+       !vec_ok ? "scalar three-pass path (unaligned or ragged rows)"
+       : cols <= 1024 ? "one warp per row, row in registers"
+       : cols <= 16384 ? "one CTA per row, row in registers"
+       : cols <= 262144 ? "one cluster per row, row in registers" : "one CTA per row, streaming passes");
   if (vec_ok && cols <= 1024) {
     const int c = (int)cols;
     if (c <= 128) launch_warp_rows<1>(x, y, rows, c, s);
