@@ -563,7 +563,7 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
       }
     }
     // shared memory must outlive every store that still reads it
-    if (lane == 0) tma_store_wait_all<0>();
+    if (lane == 0) tma_store_wait_read<0>();
     __syncwarp();
   }
 

@@ -267,8 +267,9 @@ __device__ __forceinline__ void epilogue_warp(const KernelParams& p, const CUten
     __syncwarp();
     if (lane == 0) release(acc);  // one arrival per warp
   }
-  // Shared memory must outlive every store that still reads it.
-  if (lane == 0) tma_store_wait_all<0>();
+  // Shared memory must outlive every store that still reads it (the writes themselves are complete, and visible to
+  // whatever follows in the stream, when the grid has finished).
+  if (lane == 0) tma_store_wait_read<0>();
   __syncwarp();
 }
 
@@ -348,7 +349,7 @@ __device__ __forceinline__ void epilogue_warp_gated(const KernelParams& p, const
     __syncwarp();
     if (lane == 0) release(acc);  // one arrival per warp
   }
-  if (lane == 0) tma_store_wait_all<0>();
+  if (lane == 0) tma_store_wait_read<0>();
   __syncwarp();
 }
 

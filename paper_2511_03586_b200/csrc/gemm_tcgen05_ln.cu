@@ -385,7 +385,7 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
       __syncwarp();
       if (lane < ln.cluster) mbar_arrive_cluster_relaxed(map_to_cta(consumed_bar, (uint32_t)lane));
     }
-    if (lane == 0) tma_store_wait_all<0>();
+    if (lane == 0) tma_store_wait_read<0>();
     __syncwarp();
   }
 
