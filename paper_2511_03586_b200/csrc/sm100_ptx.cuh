@@ -26,14 +26,6 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v) {
                : "memory");
 }
 
-__device__ __forceinline__ void st_shared_u32(uint32_t addr, uint32_t a) {
-  asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(a) : "memory");
-}
-__device__ __forceinline__ uint32_t ld_shared_u32(uint32_t addr) {
-  uint32_t v;
-  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
-  return v;
-}
 __device__ __forceinline__ void st_shared_f32(uint32_t addr, float a) {
   asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(a) : "memory");
 }
@@ -145,20 +137,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       }
     }
   }
-}
-
-// ---- register budget of a warpgroup ------------------------------------------
-// Every warp of a warpgroup (four consecutive warps, the first a multiple of four) executes the same one of
-// these at the same place.  A decrease returns registers to the CTA's pool at once; an increase waits until
-// the pool holds them, so the shares of all warpgroups must add up to no more than the CTA was launched with
-// (threads x registers per thread at launch).
-template <int N>
-__device__ __forceinline__ void setmaxnreg_inc() {
-  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
-}
-template <int N>
-__device__ __forceinline__ void setmaxnreg_dec() {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
 // ---- TMA (cp.async.bulk.tensor), one CTA, no multicast ----------------------
