@@ -9,10 +9,11 @@
 // six 32 KiB stages fit instead of four 48 KiB ones.
 //
 // Roles per CTA (320 threads, same as the single-CTA kernel):
-//   warp 0, one lane : TMA producer for this CTA's A rows and B half.  All byte
+//   warp 0           : TMA producer (one elected lane issues) for this CTA's A rows and B half.  All byte
 //                      counts are signalled on the EVEN CTA's "full" barrier,
-//                      which the even CTA arms for both (no multicast anywhere).
-//   warp 1, one lane : in the even CTA only, the MMA issuer (M = 256, N = 256,
+//                      which the even CTA arms for both (no load is multicast).
+//   warp 1           : in the even CTA only, the MMA issuer: the warp walks the
+//                      loop, one elected lane issues (M = 256, N = 256,
 //                      K = 16 per instruction; accumulator rows 0-127 in its own
 //                      tensor memory, rows 128-255 in the partner's).  Its
 //                      commits arrive on the "empty" / "accumulator full"
@@ -92,9 +93,12 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
-    if (lane == 0) {
-      prefetch_tensormap(&tmap_a);
-      prefetch_tensormap(&tmap_b);
+    {
+      // The whole warp walks the loop and waits; one elected lane issues the copies.
+      if (lane == 0) {
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+      }
       uint32_t it = 0;
       bool ok = true;
       for (int tile = pair; tile < p.num_tiles && ok; tile += num_pairs) {
@@ -107,18 +111,21 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
+          if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
           const uint32_t sa = smem_base + s * kStage, sb = sa + kStageA;
           const uint32_t full0 = map_to_cta(full_bar(s), 0);
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * kStage);  // bytes of both CTAs
-          tma_load_4d_pair(sa, &tmap_a, full0, kb * BK, m0, bi, bo);
-          if (B_NK) {
-            tma_load_4d_pair(sb, &tmap_b, full0, kb * BK, n0, bi, bo);
-          } else {
+          if (elect_one()) {
+            if (rank == 0) mbar_arrive_expect_tx(full_bar(s), 2 * kStage);  // bytes of both CTAs
+            tma_load_4d_pair(sa, &tmap_a, full0, kb * BK, m0, bi, bo);
+            if (B_NK) {
+              tma_load_4d_pair(sb, &tmap_b, full0, kb * BK, n0, bi, bo);
+            } else {
 #pragma unroll
-            for (int j = 0; j < kHalfN / 64; ++j)
-              tma_load_4d_pair(sb + j * (64 * BK * 2), &tmap_b, full0, n0 + j * 64, kb * BK, bi, bo);
+              for (int j = 0; j < kHalfN / 64; ++j)
+                tma_load_4d_pair(sb + j * (64 * BK * 2), &tmap_b, full0, n0 + j * 64, kb * BK, bi, bo);
+            }
           }
+          __syncwarp();
         }
       }
       if (!ok) {
@@ -131,7 +138,8 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
     }
   } else if (warp == 1) {
     // --------------------------------------------------------------- MMA issuer
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
+      // The whole warp walks the loop and waits; one elected lane issues.
       constexpr uint32_t idesc = make_idesc_bf16(2 * BM, kPairN, false, !B_NK);
       uint32_t it = 0;
       int local = 0;
@@ -139,29 +147,34 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
       for (int tile = pair; tile < p.num_tiles && ok; tile += num_pairs, ++local) {
         const int acc = local & 1;
         const uint32_t acc_ph = (local >> 1) & 1u;
-        if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc)) { ok = false; break; }
+        if (!mbar_wait_warp(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc)) { ok = false; break; }
         tcgen05_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * kPairN;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
+          if (!mbar_wait_warp(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
           tcgen05_fence_after_sync();
           const uint32_t sa = smem_base + s * kStage, sb = sa + kStageA;
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
-            const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
-                                         : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
-            mma_bf16_ss_pair(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+              const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
+              const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
+                                           : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
+              mma_bf16_ss_pair(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            mma_commit_pair(empty_bar(s), 0x3);  // the stage is free in both CTAs
           }
-          mma_commit_pair(empty_bar(s), 0x3);  // the stage is free in both CTAs
+          __syncwarp();
         }
-        if (ok) mma_commit_pair(acc_full_bar(acc), 0x3);
+        if (ok && elect_one()) mma_commit_pair(acc_full_bar(acc), 0x3);
+        __syncwarp();
       }
       if (!ok) {
         // Let every MMA already issued finish before tensor memory is freed.
-        mma_commit_pair(drain_bar, 0x1);
+        if (lane == 0) mma_commit_pair(drain_bar, 0x1);
+        __syncwarp();
         volatile int never = 0;
         mbar_wait(drain_bar, 0, &never, nullptr, 0, 20000000ull);
       }
@@ -172,7 +185,10 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
     epilogue_warp<kPairN, C_F32>(
         p, &tmap_c, tmem_base, epi_base, acc_full_bar(0), abort_flag, pair, num_pairs,
         [&](int mt) { return mt * (2 * BM) + (int)rank * BM; },
-        [&](int acc) { mbar_arrive_cluster(acc ? rel1 : rel0); });
+        // The warp's tensor-memory loads have completed (tcgen05.wait::ld) and are ordered before this signal by
+        // the tcgen05 fence; the signal publishes no memory of its own, so it carries no release ordering: a
+        // cluster-scope release here waited some 2400 clk per tile for the warp's bulk stores to drain.
+        [&](int acc) { mbar_arrive_cluster_relaxed(acc ? rel1 : rel0); });
   }
 
   // ------------------------------------------------------------------- teardown

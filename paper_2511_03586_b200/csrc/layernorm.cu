@@ -7,8 +7,11 @@
 // 128-bit loads; the mean and the centred second moment are then passes over
 // registers (data centred before squaring, mean refined by the mean of the
 // residuals: no E[x^2] - mu^2 cancellation), reduced with warp shuffles.
-//   * cols <= 1024   : one warp per row
-//   * cols <= 32768  : one CTA of 64 to 1024 threads per row
+//   * cols <= 1024   : one warp per row, two rows per CTA
+//   * cols <= 28672  : one CTA of 64 to 1024 threads per row
+//   * cols <= 262144 : one cluster of 2 to 8 CTAs per row, ceil(cols / 16384) CTAs of 512 threads up to
+//                      131072 columns and ceil(cols / 32768) of 1024 beyond (partial statistics merged
+//                      through distributed shared memory)
 //   * longer, aligned: one CTA per row, three 128-bit passes (mean from HBM; centred
 //                      second moment and normalisation from L2)
 //   * otherwise      : one CTA per row, three scalar passes from global/L2; partial
@@ -237,7 +240,7 @@ void launch_warp_rows(const float* x, const float* g, const float* b, OutT* y, i
                       cudaStream_t s) {
   constexpr int kThreads = 64, kRowsPerCta = kThreads / 32;  // two rows per CTA: the finest grain for the last, partly filled wave
   auto kernel = layernorm_rows_in_registers<VPT, 32, kThreads, OutT>;
-  // one CTA per eight rows, all launched: the hardware scheduler balances many short CTAs better than a
+  // one CTA per two rows, all launched: the hardware scheduler balances many short CTAs better than a
   // grid-stride loop over a resident set does
   const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
   const int grid = (int)(ctas < 0x7fffffff ? ctas : 0x7fffffff);

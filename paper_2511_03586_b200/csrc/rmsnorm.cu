@@ -6,7 +6,8 @@
 // HBM-bound, 8 bytes per element: the row is read once into registers with
 // 128-bit streaming loads, the sum of squares is reduced with warp shuffles (and
 // through shared memory when several warps share a row), and the row is written
-// once.  Same paths as the LayerNorm kernel: a warp, a CTA or a cluster of CTAs per row, by row length.
+// once.  Same paths as the LayerNorm kernel: a warp (cols <= 1024), a CTA (<= 32768) or a cluster of 2 to 8
+// CTAs (<= 262144) per row, by row length.
 #include "pd_common.cuh"
 
 namespace pd {

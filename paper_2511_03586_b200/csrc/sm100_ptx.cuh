@@ -1,5 +1,7 @@
 // Inline-PTX wrappers for the Blackwell (sm_100a) data path used by the
-// tensor-core kernels: mbarriers, TMA tensor copies (never multicast), tensor
+// tensor-core kernels: mbarriers, TMA tensor copies (no TMA or bulk load uses
+// multicast; the only .multicast::cluster is the arrival of a CTA pair's
+// tcgen05.commit on both CTAs' mbarriers, in this GPU's own shared memory), tensor
 // memory management and tcgen05 MMA / load instructions, plus the shared-memory
 // and instruction descriptors the MMA consumes.  Internal to the library.
 #pragma once
@@ -13,6 +15,22 @@ namespace sm100 {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// True in exactly one lane of a fully converged warp.  The roles that issue tcgen05.mma run their loops with the
+// whole warp (so that barrier addresses, descriptors and counters stay warp-uniform values) and elect one lane
+// for the instructions themselves: with a single lane in a divergent branch the same loop took so many more
+// issue slots that busy epilogue warps on the same scheduler visibly delayed the products.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "elect.sync _|p, 0xffffffff;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(pred));
+  return pred != 0;
 }
 
 __device__ __forceinline__ uint64_t global_timer_ns() {
@@ -137,6 +155,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       }
     }
   }
+}
+
+// The same wait made by all 32 lanes of a converged warp, with one answer for the warp: false when any lane gave up.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                               int code, uint64_t limit_ns = 2000000000ull) {
+  return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, status, code, limit_ns));
 }
 
 // ---- TMA (cp.async.bulk.tensor), one CTA, no multicast ----------------------
@@ -313,11 +337,9 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
 }
-// Arrive on an mbarrier given by a shared::cluster address (possibly in the peer CTA).
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// The same without memory ordering: for signals that publish no data of their own.
+// Arrive on an mbarrier given by a shared::cluster address (possibly in the peer CTA), without memory ordering:
+// for signals that publish no data of their own (a release at cluster scope first waits for everything the
+// thread has written, its bulk stores included).
 __device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }

@@ -5,10 +5,11 @@
 // HBM-bound: 8 bytes per element (4 when writing bf16).  Each row is read from
 // global memory exactly once into registers with 128-bit loads, reduced with
 // warp shuffles, and written once.
-//   * cols <= 1024            : one warp per row (up to 8 float4 per lane)
-//   * cols <= 32768           : one CTA of 64 to 1024 threads per row (8 float4 per thread)
-//   * cols <= 262144          : one cluster of 2, 4 or 8 such CTAs per row (statistics combined through
-//                               distributed shared memory)
+//   * cols <= 1024            : one warp per row (up to 8 float4 per lane), two rows per CTA
+//   * cols <= 16384           : one CTA of 64 to 512 threads per row (8 float4 per thread)
+//   * cols <= 262144          : one cluster of 2 to 8 CTAs per row, ceil(cols / 16384) CTAs of 512 threads up
+//                               to 131072 columns and ceil(cols / 32768) of 1024 beyond (statistics combined
+//                               through distributed shared memory)
 //   * longer, 16-byte aligned : one CTA per row, online (max, sum) pass from HBM, normalising pass from L2
 //   * anything else / ragged  : one CTA per row, three scalar passes from global/L2
 #include "pd_common.cuh"
@@ -168,7 +169,7 @@ template <int VPT, typename OutT>
 void launch_warp_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStream_t s) {
   constexpr int kThreads = 64, kRowsPerCta = kThreads / 32;  // two rows per CTA: the finest grain for the last, partly filled wave
   auto kernel = softmax_rows_in_registers<VPT, 32, kThreads, OutT>;
-  // one CTA per eight rows, all launched: the hardware scheduler balances many short CTAs better than a
+  // one CTA per two rows, all launched: the hardware scheduler balances many short CTAs better than a
   // grid-stride loop over a resident set does
   const int64_t ctas = (rows + kRowsPerCta - 1) / kRowsPerCta;
   const int grid = (int)(ctas < 0x7fffffff ? ctas : 0x7fffffff);
@@ -202,8 +203,7 @@ pd_status dispatch(const float* x, OutT* y, int64_t rows, int64_t cols, cudaStre
     if (c <= 2048) launch_cta_rows<64>(x, y, rows, c, s);
     else if (c <= 4096) launch_cta_rows<128>(x, y, rows, c, s);
     else if (c <= 8192) launch_cta_rows<256>(x, y, rows, c, s);
-    else if (c <= 16384) launch_cta_rows<512>(x, y, rows, c, s);
-    else launch_cta_rows<1024>(x, y, rows, c, s);
+    else launch_cta_rows<512>(x, y, rows, c, s);
   } else if (vec_ok && cols <= 262144 && rows * 8 <= 0x7fffffff) {
     if (cols <= 131072) {
       const unsigned cl = (unsigned)((cols + 16383) / 16384);
