@@ -5,7 +5,7 @@
 // on the packed projection qkv[tokens, 3*hidden] = [Q | K | V].  Scores and
 // probabilities never leave the SM.
 //
-// One persistent CTA of 512 threads per SM walks over work units of (batch,
+// One persistent CTA of 544 threads per SM walks over work units of (batch,
 // head, pair of 128-query blocks).  K and V of the head (up to 512 x 64 each)
 // sit in shared memory in four chunks of 128 keys, each with its own full and
 // empty barrier, so that the next unit's chunks stream in while the current
@@ -16,14 +16,17 @@
 // tensor memory (all 512 columns), so that the tensor core, the exponential
 // unit and the barrier round trips overlap, also across unit boundaries.
 //
-//   warp 8, lane 16  : TMA producer (per unit: Q of each slot, then the K and V
+//   warp 16          : TMA producer (per unit: Q of each slot, then the K and V
 //                      chunks in the order the previous unit releases them).
-//   warps 8, 10      : score issuers, one thread per slot, each in a warp of
-//                      its own (see kScoreWarp0 below): for block g of
+//                      Like the issuers below, the whole warp walks the loop
+//                      and waits, so that its addresses and counters stay
+//                      warp-uniform values, and one elected lane issues.
+//   warps 8, 10      : score issuers, one warp per slot
+//                      (see kScoreWarp0 below): for block g of
 //                      64 keys S = Q K_g^T (128 x 64 x 64) into one of the slot's
 //                      two score buffers, as soon as the softmax warps have
 //                      read that buffer's previous contents.
-//   warps 9, 11      : output issuers, one thread per slot: when the
+//   warps 9, 11      : output issuers, one warp per slot: when the
 //                      slot's softmax warps have published P_g,
 //                      O += P_g V_g (128 x 64 x 64) into the slot's 64 output
 //                      columns, P_g read from tensor memory as the A operand.
@@ -67,18 +70,19 @@ constexpr int kBlockQ = 128;      // queries per slot = TMEM lanes
 constexpr int kBlockK = 64;       // keys per score block
 constexpr int kMaxKeys = 512;
 constexpr int kSlots = 2;         // query blocks in flight
-constexpr int kThreads = 512;
+constexpr int kThreads = 544;
 constexpr int kSlotThreads = 128, kSlotWarps = kSlotThreads / 32;
-// warps 0-7 softmax, 8-11 the four MMA-issuing threads, 12-15 epilogue (sixteen warps: 128 registers a thread).
+// warps 0-7 softmax, 8-11 the four MMA-issuing warps, 12-15 epilogue, 16 the TMA producer (seventeen warps: 120 registers a thread).
 // Every tcgen05.mma / tcgen05.commit issuing thread has a warp of its own: two lanes of one warp that reach the
 // same tcgen05 instruction together, with different operands, do not get two independent operations (attention
 // with peaked rows came out wrong that way whenever the two slots drifted apart).  The TMA producer issues no
 // tcgen05 instruction and rides along as another lane of the first issuer's warp.
 constexpr int kScoreWarp0 = 8, kOutputWarp0 = 9, kScoreWarp1 = 10, kOutputWarp1 = 11;
-constexpr int kProducerWarp = kScoreWarp0, kProducerLane = 16;
+constexpr int kProducerWarp = 16;
 constexpr int kEpilogueWarp0 = 12;  // warp w reads the tensor-memory lanes 32 * (w % 4) ... + 31
 constexpr int kAllocWarp = kOutputWarp0;
-static_assert(kEpilogueWarp0 % 4 == 0 && kThreads == 32 * (kEpilogueWarp0 + 4), "epilogue warps cover the four lane quarters");
+static_assert(kEpilogueWarp0 % 4 == 0 && kProducerWarp == kEpilogueWarp0 + 4 && kThreads == 32 * (kProducerWarp + 1),
+              "epilogue warps cover the four lane quarters; the producer warp comes last");
 
 constexpr int kSmemK = kMaxKeys * kD * 2;        // 64 KiB
 constexpr int kSmemV = kMaxKeys * kD * 2;        // 64 KiB
@@ -204,27 +208,34 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
   const int G = p.k_blocks;
   const int NC = (G + 1) >> 1;  // chunks of 128 keys in use; chunk c holds score blocks 2c and 2c + 1
 
-  if (warp == kProducerWarp && lane == kProducerLane) {
+  if (warp == kProducerWarp) {
     // ------------------------------------------------------------- TMA producer
     // Per unit: the two query tiles (into the slot's other buffer, normally free long before), then the chunks
     // of K and V in the order in which the previous unit releases them.
+    // The whole warp walks the loop and waits; one elected lane issues the copies.
     {
-      prefetch_tensormap(&tmap_q); prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v);
+      if (lane == 0) { prefetch_tensormap(&tmap_q); prefetch_tensormap(&tmap_k); prefetch_tensormap(&tmap_v); }
       uint32_t n_unit = 0, n_q[kSlots] = {0, 0};
       uint32_t armed_k = 0, armed_v = 0;  // bit c: chunk c of the current unit has been requested
       bool ok = true;
       auto load_k = [&](int c, int h, int b) {
         if (c >= NC || !ok) return;
-        if (!mbar_wait(k_empty(c), (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; return; }
-        mbar_arrive_expect_tx(k_full(c), kSmemChunk);
-        tma_load_4d(sK + c * kSmemChunk, &tmap_k, k_full(c), 0, c * kChunkKeys, h, b);
+        if (!mbar_wait_warp(k_empty(c), (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; return; }
+        if (elect_one()) {
+          mbar_arrive_expect_tx(k_full(c), kSmemChunk);
+          tma_load_4d(sK + c * kSmemChunk, &tmap_k, k_full(c), 0, c * kChunkKeys, h, b);
+        }
+        __syncwarp();
         armed_k |= 1u << c;
       };
       auto load_v = [&](int c, int h, int b) {
         if (c >= NC || !ok) return;
-        if (!mbar_wait(v_empty(c), (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; return; }
-        mbar_arrive_expect_tx(v_full(c), kSmemChunk);
-        tma_load_4d(sV + c * kSmemChunk, &tmap_v, v_full(c), 0, c * kChunkKeys, h, b);
+        if (!mbar_wait_warp(v_empty(c), (n_unit & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; return; }
+        if (elect_one()) {
+          mbar_arrive_expect_tx(v_full(c), kSmemChunk);
+          tma_load_4d(sV + c * kSmemChunk, &tmap_v, v_full(c), 0, c * kChunkKeys, h, b);
+        }
+        __syncwarp();
         armed_v |= 1u << c;
       };
       for (int unit = blockIdx.x; unit < p.num_units && ok; unit += gridDim.x, ++n_unit) {
@@ -233,10 +244,13 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         armed_k = armed_v = 0;
         for (int s = 0; s < nslots && ok; ++s) {
           const uint32_t qb = n_q[s] & 1u; const uint32_t qpar = ((n_q[s] >> 1) & 1u) ^ 1u;
-          if (!mbar_wait(q_empty(s, qb), qpar, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
+          if (!mbar_wait_warp(q_empty(s, qb), qpar, abort_flag, p.status, kTimeoutAttnProducer)) { ok = false; break; }
           ++n_q[s];
-          mbar_arrive_expect_tx(q_full(s, qb), kSmemQ);
-          tma_load_4d(sQ + (2 * s + qb) * kSmemQ, &tmap_q, q_full(s, qb), 0, (qb0 + s) * kBlockQ, h, b);
+          if (elect_one()) {
+            mbar_arrive_expect_tx(q_full(s, qb), kSmemQ);
+            tma_load_4d(sQ + (2 * s + qb) * kSmemQ, &tmap_q, q_full(s, qb), 0, (qb0 + s) * kBlockQ, h, b);
+          }
+          __syncwarp();
         }
         load_k(0, h, b); load_k(1, h, b); load_v(0, h, b); load_k(2, h, b); load_v(1, h, b); load_k(3, h, b);
         load_v(2, h, b); load_v(3, h, b);
@@ -259,8 +273,8 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
       }
     }
   } else if (warp == kScoreWarp0 || warp == kScoreWarp1) {
-    // ---------------------- score-product issuers: one thread per slot, each in its own warp
-    if (lane == 0) {
+    // ---------------------- score-product issuers: one warp per slot walks the loop, one elected lane issues
+    {
       const int s = warp == kScoreWarp0 ? 0 : 1;
       constexpr uint32_t idesc_s = make_idesc_bf16(kBlockQ, kBlockK, false, false);  // Q K^T: both K-major
       const uint64_t k_desc = make_smem_desc(sK, 0, 1024);
@@ -274,39 +288,45 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         const uint32_t qb = n_q & 1u; const uint32_t qpar = (n_q >> 1) & 1u;
         uint64_t q_desc = 0;
         if (active) {
-          if (!mbar_wait(q_full(s, qb), qpar, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+          if (!mbar_wait_warp(q_full(s, qb), qpar, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
           ++n_q;
           q_desc = make_smem_desc(sQ + (2 * s + qb) * kSmemQ, 0, 1024);
         }
         for (int c = 0; c < NC && ok; ++c) {
-          if (!mbar_wait(k_full(c), n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+          if (!mbar_wait_warp(k_full(c), n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
           if (active) {
             for (int g = 2 * c; g < min(2 * c + 2, G); ++g, ++t) {
               const uint32_t buf = t & 1u;
-              if (!mbar_wait(s_empty(s, buf), ((t >> 1) & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+              if (!mbar_wait_warp(s_empty(s, buf), ((t >> 1) & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
               tcgen05_fence_after_sync();
               const uint64_t kg = k_desc + (uint64_t)(g * ((kBlockK * 128) >> 4));
+              if (elect_one()) {
 #pragma unroll
-              for (int ks = 0; ks < kD / 16; ++ks)
-                mma_bf16_ss(d_tmem + buf * kBlockK, q_desc + 2 * ks, kg + 2 * ks, idesc_s, ks != 0 ? 1u : 0u);
-              mma_commit(s_full(s, buf));
+                for (int ks = 0; ks < kD / 16; ++ks)
+                  mma_bf16_ss(d_tmem + buf * kBlockK, q_desc + 2 * ks, kg + 2 * ks, idesc_s, ks != 0 ? 1u : 0u);
+                mma_commit(s_full(s, buf));
+              }
+              __syncwarp();
             }
             if (!ok) break;
           }
-          mma_commit(k_empty(c));  // both score issuers arrive, whether or not their slot is in use
+          if (elect_one()) mma_commit(k_empty(c));  // both score issuers arrive, whether or not their slot is in use
+          __syncwarp();
         }
         if (!ok) break;
-        if (active) mma_commit(q_empty(s, qb));
+        if (active && elect_one()) mma_commit(q_empty(s, qb));
+        __syncwarp();
       }
       if (!ok) {
-        mma_commit(drain_bar + 16u + 8u * s);
+        if (lane == 0) mma_commit(drain_bar + 16u + 8u * s);
+        __syncwarp();
         volatile int never = 0;
         mbar_wait(drain_bar + 16u + 8u * s, 0, &never, nullptr, 0, 20000000ull);
       }
     }
   } else if (warp == kOutputWarp0 || warp == kOutputWarp1) {
-    // ------------------------ P V product issuers: one thread per slot, each in its own warp
-    if (lane == 0) {
+    // ------------------------ P V product issuers: one warp per slot walks the loop, one elected lane issues
+    {
       const int s = warp == kOutputWarp0 ? 0 : 1;
       constexpr uint32_t idesc_o = make_idesc_bf16(kBlockQ, kD, false, true);  // V is MN-major
       const uint64_t v_desc = make_smem_desc(sV, 0, 1024);
@@ -319,35 +339,41 @@ attention_fwd_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_q, const _
         const bool active = s < nslots;
         if (active) {
           // the previous unit's output of this slot must have been read before it is overwritten
-          if (!mbar_wait(o_empty(s), (n_us & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+          if (!mbar_wait_warp(o_empty(s), (n_us & 1u) ^ 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
         }
         for (int c = 0; c < NC && ok; ++c) {
-          if (!mbar_wait(v_full(c), n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+          if (!mbar_wait_warp(v_full(c), n_unit & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
           if (active) {
             for (int g = 2 * c; g < min(2 * c + 2, G); ++g, ++t) {
               const uint32_t buf = t & 1u;
-              if (!mbar_wait(p_full(s, buf), (t >> 1) & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
+              if (!mbar_wait_warp(p_full(s, buf), (t >> 1) & 1u, abort_flag, p.status, kTimeoutAttnMma)) { ok = false; break; }
               tcgen05_fence_after_sync();
               // P_g is the A operand straight from tensor memory: keys 2j, 2j + 1 of the block in column j
               const uint32_t pg = tmem_base + kTmemP + s * 64 + buf * 32;
               const uint64_t vg = v_desc + (uint64_t)(g * ((kBlockK * 128) >> 4));
+              if (elect_one()) {
 #pragma unroll
-              for (int ks = 0; ks < kBlockK / 16; ++ks)
-                mma_bf16_ts(d_tmem, pg + 8 * ks, vg + ks * ((16 * 128) >> 4), idesc_o, (g | ks) != 0 ? 1u : 0u);
-              mma_commit(p_empty(s, buf));
+                for (int ks = 0; ks < kBlockK / 16; ++ks)
+                  mma_bf16_ts(d_tmem, pg + 8 * ks, vg + ks * ((16 * 128) >> 4), idesc_o, (g | ks) != 0 ? 1u : 0u);
+                mma_commit(p_empty(s, buf));
+              }
+              __syncwarp();
             }
             if (!ok) break;
           }
-          mma_commit(v_empty(c));  // both output issuers arrive
+          if (elect_one()) mma_commit(v_empty(c));  // both output issuers arrive
+          __syncwarp();
         }
         if (!ok) break;
         if (active) {
-          mma_commit(o_full(s));
+          if (elect_one()) mma_commit(o_full(s));
+          __syncwarp();
           ++n_us;
         }
       }
       if (!ok) {
-        mma_commit(drain_bar + 8u * s);
+        if (lane == 0) mma_commit(drain_bar + 8u * s);
+        __syncwarp();
         volatile int never = 0;
         mbar_wait(drain_bar + 8u * s, 0, &never, nullptr, 0, 20000000ull);
       }

@@ -3,10 +3,10 @@
 //   C[m,n] = act(alpha * sum_k A[m,k] B[k,n] + bias[n]) + residual[m,n]
 //
 // Persistent, warp-specialised kernel, one CTA of 320 threads per SM:
-//   warp 0, one lane : TMA producer.  Streams 128 x 64 tiles of A and BN x 64
+//   warp 0           : TMA producer (the warp walks the loop, one elected lane issues).  Streams 128 x 64 tiles of A and BN x 64
 //                      tiles of B (128-byte swizzle) into a ring of shared-memory
 //                      stages; a "full" mbarrier per stage counts the bytes.
-//   warp 1, one lane : MMA issuer.  Four tcgen05.mma (128 x BN x 16) per stage
+//   warp 1           : MMA issuer (likewise).  Four tcgen05.mma (128 x BN x 16) per stage
 //                      accumulate into one of two TMEM accumulators; a
 //                      tcgen05.commit hands the stage back ("empty" barrier) and,
 //                      after the last k-block, publishes the accumulator.
@@ -101,10 +101,13 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
-    if (lane == 0) {
-      prefetch_tensormap(&tmap_a);
-      prefetch_tensormap(&tmap_b);
-      if (GATED) prefetch_tensormap(&tmap_b2);
+    {
+      // The whole warp walks the loop and waits; one elected lane issues the copies.
+      if (lane == 0) {
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+        if (GATED) prefetch_tensormap(&tmap_b2);
+      }
       uint32_t it = 0;  // k-blocks issued so far, over all tiles
       bool ok = true;
       // (test switch: with withhold_loads set the producer issues nothing, and the wait for the first stage runs out)
@@ -116,22 +119,25 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer, wait_limit(p))) { ok = false; break; }
+          if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer, wait_limit(p))) { ok = false; break; }
           const uint32_t sa = smem_base + s * C::kStage, sb = sa + C::kStageA;
-          mbar_arrive_expect_tx(full_bar(s), C::kStage);
-          tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, bi, bo);
-          if constexpr (GATED) {
+          if (elect_one()) {
+            mbar_arrive_expect_tx(full_bar(s), C::kStage);
+            tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, bi, bo);
+            if constexpr (GATED) {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j)
-              tma_load_4d(sb + j * (64 * BK * 2), j < BN / 128 ? &tmap_b : &tmap_b2, full_bar(s),
-                          nt * (BN / 2) + (j % (BN / 128)) * 64, kb * BK, 0, 0);
-          } else if (B_NK) {
-            tma_load_4d(sb, &tmap_b, full_bar(s), kb * BK, nt * BN, bi, bo);
-          } else {
+              for (int j = 0; j < BN / 64; ++j)
+                tma_load_4d(sb + j * (64 * BK * 2), j < BN / 128 ? &tmap_b : &tmap_b2, full_bar(s),
+                            nt * (BN / 2) + (j % (BN / 128)) * 64, kb * BK, 0, 0);
+            } else if (B_NK) {
+              tma_load_4d(sb, &tmap_b, full_bar(s), kb * BK, nt * BN, bi, bo);
+            } else {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j)
-              tma_load_4d(sb + j * (64 * BK * 2), &tmap_b, full_bar(s), nt * BN + j * 64, kb * BK, bi, bo);
+              for (int j = 0; j < BN / 64; ++j)
+                tma_load_4d(sb + j * (64 * BK * 2), &tmap_b, full_bar(s), nt * BN + j * 64, kb * BK, bi, bo);
+            }
           }
+          __syncwarp();
         }
       }
       if (!ok) {
@@ -147,7 +153,8 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     }
   } else if (warp == 1) {
     // --------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    {
+      // The whole warp walks the loop and waits; one elected lane issues.
       constexpr uint32_t idesc = make_idesc_bf16(BM, BN, false, !B_NK);
       uint32_t it = 0;
       int local = 0;
@@ -155,29 +162,34 @@ gemm_bf16_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       for (int tile = blockIdx.x; tile < p.num_tiles && ok; tile += gridDim.x, ++local) {
         const int acc = local & 1;
         const uint32_t acc_ph = (local >> 1) & 1u;
-        if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc, wait_limit(p))) { ok = false; break; }
+        if (!mbar_wait_warp(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc, wait_limit(p))) { ok = false; break; }
         tcgen05_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull, wait_limit(p))) { ok = false; break; }
+          if (!mbar_wait_warp(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull, wait_limit(p))) { ok = false; break; }
           tcgen05_fence_after_sync();
           const uint32_t sa = smem_base + s * C::kStage, sb = sa + C::kStageA;
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
-            const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
-                                         : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
-            mma_bf16_ss(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+              const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
+              const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
+                                           : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
+              mma_bf16_ss(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            mma_commit(empty_bar(s));
           }
-          mma_commit(empty_bar(s));
+          __syncwarp();
         }
-        if (ok) mma_commit(acc_full_bar(acc));
+        if (ok && elect_one()) mma_commit(acc_full_bar(acc));
+        __syncwarp();
       }
       if (!ok) {
         // Let every MMA already issued finish before tensor memory is freed.
-        mma_commit(drain_bar);
+        if (lane == 0) mma_commit(drain_bar);
+        __syncwarp();
         volatile int never = 0;
         mbar_wait(drain_bar, 0, &never, nullptr, 0, 20000000ull);
       }

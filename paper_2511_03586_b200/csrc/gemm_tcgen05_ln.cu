@@ -4,8 +4,8 @@
 // LayerNorm needs whole rows, a 128 x 256 accumulator tile holds a quarter of a
 // 1024-wide row.  So the N / 256 CTAs that own the tiles of the same 128 rows
 // form a thread-block cluster and run in lockstep over the row blocks:
-//   * main loop: as in the single-CTA GEMM (TMA producer lane, MMA issuer lane,
-//     two TMEM accumulators, four 48 KiB stages);
+//   * main loop: as in the single-CTA GEMM (TMA producer warp, MMA issuer warp,
+//     one elected lane of each issuing; two TMEM accumulators, four 48 KiB stages);
 //   * epilogue pass 1 (sixteen warps, so that four per scheduler hide each
 //     other's latencies): every epilogue thread owns 64 columns of one row.  It
 //     forms v = acc + bias + residual in fp32, writes v back over the
@@ -128,9 +128,12 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
-    if (lane == 0) {
-      prefetch_tensormap(&tmap_a);
-      prefetch_tensormap(&tmap_b);
+    {
+      // The whole warp walks the loop and waits; one elected lane issues the copies.
+      if (lane == 0) {
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+      }
       uint32_t it = 0;
       bool ok = true;
       for (int lt = cluster_id; lt < p.tiles_m && ok; lt += num_clusters) {
@@ -138,17 +141,20 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
+          if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
           const uint32_t sa = smem_base + s * kStage, sb = sa + kStageA;
-          mbar_arrive_expect_tx(full_bar(s), kStage);
-          tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, 0, 0);
-          if (B_NK) {
-            tma_load_4d(sb, &tmap_b, full_bar(s), kb * BK, nt * BN, 0, 0);
-          } else {
+          if (elect_one()) {
+            mbar_arrive_expect_tx(full_bar(s), kStage);
+            tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, 0, 0);
+            if (B_NK) {
+              tma_load_4d(sb, &tmap_b, full_bar(s), kb * BK, nt * BN, 0, 0);
+            } else {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j)
-              tma_load_4d(sb + j * (64 * BK * 2), &tmap_b, full_bar(s), nt * BN + j * 64, kb * BK, 0, 0);
+              for (int j = 0; j < BN / 64; ++j)
+                tma_load_4d(sb + j * (64 * BK * 2), &tmap_b, full_bar(s), nt * BN + j * 64, kb * BK, 0, 0);
+            }
           }
+          __syncwarp();
         }
       }
       if (!ok) {
@@ -163,7 +169,8 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
     }
   } else if (warp == 1) {
     // --------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    {
+      // The whole warp walks the loop and waits; one elected lane issues.
       constexpr uint32_t idesc = make_idesc_bf16(BM, BN, false, !B_NK);
       uint32_t it = 0;
       int local = 0;
@@ -171,28 +178,33 @@ gemm_bias_residual_layernorm_kernel(const __grid_constant__ CUtensorMap tmap_a,
       for (int lt = cluster_id; lt < p.tiles_m && ok; lt += num_clusters, ++local) {
         const int acc = local & 1;
         const uint32_t acc_ph = (local >> 1) & 1u;
-        if (!mbar_wait(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc)) { ok = false; break; }
+        if (!mbar_wait_warp(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc)) { ok = false; break; }
         tcgen05_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
+          if (!mbar_wait_warp(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
           tcgen05_fence_after_sync();
           const uint32_t sa = smem_base + s * kStage, sb = sa + kStageA;
+          if (elect_one()) {
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k) {
-            const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
-            const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
-                                         : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
-            mma_bf16_ss(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+              const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
+              const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
+                                           : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
+              mma_bf16_ss(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            mma_commit(empty_bar(s));
           }
-          mma_commit(empty_bar(s));
+          __syncwarp();
         }
-        if (ok) mma_commit(acc_full_bar(acc));
+        if (ok && elect_one()) mma_commit(acc_full_bar(acc));
+        __syncwarp();
       }
       if (!ok) {
-        mma_commit(drain_bar);
+        if (lane == 0) mma_commit(drain_bar);
+        __syncwarp();
         volatile int never = 0;
         mbar_wait(drain_bar, 0, &never, nullptr, 0, 20000000ull);
       }

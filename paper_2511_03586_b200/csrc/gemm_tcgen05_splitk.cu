@@ -95,31 +95,37 @@ gemm_bf16_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a, cons
   bool acc_ok = true;  // epilogue warps: this CTA's accumulator is complete
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
-    if (lane == 0) {
-      prefetch_tensormap(&tmap_a);
-      prefetch_tensormap(&tmap_b);
-      if (GATED) prefetch_tensormap(&tmap_b2);
+    {
+      // The whole warp walks the loop and waits; one elected lane issues the copies.
+      if (lane == 0) {
+        prefetch_tensormap(&tmap_a);
+        prefetch_tensormap(&tmap_b);
+        if (GATED) prefetch_tensormap(&tmap_b2);
+      }
       uint32_t it = 0;
       bool ok = true;
       for (int kb = kb0; kb < kb1; ++kb, ++it) {
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
+        if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
         const uint32_t sa = smem_base + s * C::kStage, sb = sa + C::kStageA;
-        mbar_arrive_expect_tx(full_bar(s), C::kStage);
-        tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, 0, 0);
-        if constexpr (GATED) {
+        if (elect_one()) {
+          mbar_arrive_expect_tx(full_bar(s), C::kStage);
+          tma_load_4d(sa, &tmap_a, full_bar(s), kb * BK, mt * BM, 0, 0);
+          if constexpr (GATED) {
 #pragma unroll
-          for (int j = 0; j < BN / 64; ++j)
-            tma_load_4d(sb + j * (64 * BK * 2), j < BN / 128 ? &tmap_b : &tmap_b2, full_bar(s),
-                        nt * OC + (j % (BN / 128)) * 64, kb * BK, 0, 0);
-        } else if (B_NK) {
-          tma_load_4d(sb, &tmap_b, full_bar(s), kb * BK, nt * BN, 0, 0);
-        } else {
+            for (int j = 0; j < BN / 64; ++j)
+              tma_load_4d(sb + j * (64 * BK * 2), j < BN / 128 ? &tmap_b : &tmap_b2, full_bar(s),
+                          nt * OC + (j % (BN / 128)) * 64, kb * BK, 0, 0);
+          } else if (B_NK) {
+            tma_load_4d(sb, &tmap_b, full_bar(s), kb * BK, nt * BN, 0, 0);
+          } else {
 #pragma unroll
-          for (int j = 0; j < BN / 64; ++j)
-            tma_load_4d(sb + j * (64 * BK * 2), &tmap_b, full_bar(s), nt * BN + j * 64, kb * BK, 0, 0);
+            for (int j = 0; j < BN / 64; ++j)
+              tma_load_4d(sb + j * (64 * BK * 2), &tmap_b, full_bar(s), nt * BN + j * 64, kb * BK, 0, 0);
+          }
         }
+        __syncwarp();
       }
       if (!ok) {
         const uint32_t issued = it;
@@ -133,29 +139,35 @@ gemm_bf16_splitk_cluster_kernel(const __grid_constant__ CUtensorMap tmap_a, cons
     }
   } else if (warp == 1) {
     // --------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    {
+      // The whole warp walks the loop and waits; one elected lane issues.
       constexpr uint32_t idesc = make_idesc_bf16(BM, BN, false, !B_NK);
       uint32_t it = 0;
       bool ok = true;
       for (int kb = kb0; kb < kb1; ++kb, ++it) {
         const int s = it % kStages;
         const uint32_t ph = (it / kStages) & 1u;
-        if (!mbar_wait(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
+        if (!mbar_wait_warp(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
         tcgen05_fence_after_sync();
         const uint32_t sa = smem_base + s * C::kStage, sb = sa + C::kStageA;
+        if (elect_one()) {
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; ++k) {
-          const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
-          const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
-                                       : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
-          mma_bf16_ss(tmem_base, a_desc, b_desc, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            const uint64_t a_desc = make_smem_desc(sa + k * (UMMA_K * 2), 0, 1024);
+            const uint64_t b_desc = B_NK ? make_smem_desc(sb + k * (UMMA_K * 2), 0, 1024)
+                                         : make_smem_desc(sb + k * (UMMA_K * 128), 64 * BK * 2, 1024);
+            mma_bf16_ss(tmem_base, a_desc, b_desc, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          }
+          mma_commit(empty_bar(s));
         }
-        mma_commit(empty_bar(s));
+        __syncwarp();
       }
       if (ok) {
-        mma_commit(acc_full_bar);
+        if (elect_one()) mma_commit(acc_full_bar);
+        __syncwarp();
       } else {
-        mma_commit(drain_bar);
+        if (lane == 0) mma_commit(drain_bar);
+        __syncwarp();
         volatile int never = 0;
         mbar_wait(drain_bar, 0, &never, nullptr, 0, 20000000ull);
       }
