@@ -121,6 +121,34 @@ def test_repeatable_and_matches_unfused_kernels(api):
     assert max_rel_floored(host(y1), host(z)) < TOL_ONE_ROUNDING
 
 
+def test_graph_replay_and_changing_cluster_sizes(api):
+    # Launches of different shapes (clusters of 4, 1, 8 and 2 CTAs) captured into one CUDA graph and replayed give
+    # the eager results every time.
+    shapes = [(1500, 1024, 128), (700, 256, 64), (520, 2048, 64), (3000, 512, 192)]
+    ps = [inputs.gemm_layernorm_inputs(M, N, K, seed=11 + i) for i, (M, N, K) in enumerate(shapes)]
+    args = [(dev_bf16(p["a_bits"]), dev_bf16(p["b_bits"]), dev_f32(p["bias"]), dev_bf16(p["residual_bits"]),
+             dev_f32(p["gamma"]), dev_f32(p["beta"]), p["eps"]) for p in ps]
+    eager = [api.pd_gemm_bias_residual_layernorm(*a) for a in args]
+    for p, y in zip(ps, eager):
+        assert max_rel_floored(host(y), _oracle(p)) < TOL_ONE_ROUNDING
+    outs = [torch.empty_like(y) for y in eager]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for a, o in zip(args, outs):
+                api.pd_gemm_bias_residual_layernorm(*a, y=o)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        for y, o in zip(eager, outs):
+            assert torch.equal(y, o)
+
+
 def test_argument_errors(api):
     from paper_2511_03586_b200.api import PdError
     p = inputs.gemm_layernorm_inputs(64, 256, 64, seed=0)
