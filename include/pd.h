@@ -80,12 +80,15 @@ pd_status pd_clear_device_status(void);
  * 4.3 "Search with PerfLLM": a candidate that does not finish is cut off and
  * reported, it does not take the system down).
  * pd_debug_set_wait_limit_ns: the time after which a wait inside the single-CTA
- * contraction kernel (pd_set_gemm_tile_mode(1)) gives up, 1 us to 10 s (else
- * PD_ERR_BAD_SHAPE); default 2 s.  pd_debug_withhold_loads(1): that kernel's
- * producer thread issues no load, so the thread that feeds the tensor core
- * waits for its first operand stage in vain, gives up after the limit, records
- * code 102 in the device status word, and every role of the kernel drains and
- * returns (nothing faults, traps or stays behind; the output is not written).
+ * and the CTA-pair contraction kernels (pd_set_gemm_tile_mode(1) / (2)) gives
+ * up, 1 us to 10 s (else PD_ERR_BAD_SHAPE); default 2 s.
+ * pd_debug_withhold_loads(1): those kernels' producers issue no load, so the
+ * warp that feeds the tensor core waits for its first operand stage in vain,
+ * gives up after the limit, records code 102 in the device status word, and
+ * every role of the kernel drains and returns (in the pair kernel the partner
+ * CTA's epilogue warps give up on their own wait for the accumulator, code
+ * 104 if they are first; nothing faults, traps or stays behind; the output is
+ * not written).
  * pd_debug_withhold_loads(0) restores normal operation.  Both settings are
  * process-wide and apply to launches enqueued after the call. */
 pd_status pd_debug_set_wait_limit_ns(uint64_t limit_ns);

@@ -29,8 +29,9 @@ struct KernelParams {
   int tiles_m, tiles_n, batch_inner, num_tiles;  // num_tiles = batch_outer * batch_inner * tiles_m * tiles_n
   float alpha;
   int c_is_f32, act;  // act: 0 nothing, 1 erf-form GELU, 2 ReLU
-  // Single-CTA kernel only (zero elsewhere): the time after which its waits give up (0: the default of 2 s), and
-  // the test switch that makes its producer skip every load, so that the wait for the first stage runs out.
+  // Single-CTA and CTA-pair kernels only (zero elsewhere): the time after which their waits give up (0: the default
+  // of 2 s), and the test switch that makes their producers skip every load, so that the wait for the first stage
+  // runs out.
   unsigned long long wait_limit_ns;
   int withhold_loads;
 };

@@ -101,7 +101,8 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
       }
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = pair; tile < p.num_tiles && ok; tile += num_pairs) {
+      // (test switch: with withhold_loads set the producer issues nothing, and the wait for the first stage runs out)
+      for (int tile = pair; tile < p.num_tiles && ok && !p.withhold_loads; tile += num_pairs) {
         const int nt = tile % p.tiles_n;
         const int mt = (tile / p.tiles_n) % p.tiles_m;
         const int b = tile / (p.tiles_n * p.tiles_m);
@@ -111,7 +112,7 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer)) { ok = false; break; }
+          if (!mbar_wait_warp(empty_bar(s), ph ^ 1u, abort_flag, p.status, kTimeoutProducer, wait_limit(p))) { ok = false; break; }
           const uint32_t sa = smem_base + s * kStage, sb = sa + kStageA;
           const uint32_t full0 = map_to_cta(full_bar(s), 0);
           if (elect_one()) {
@@ -147,13 +148,13 @@ gemm_bf16_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const 
       for (int tile = pair; tile < p.num_tiles && ok; tile += num_pairs, ++local) {
         const int acc = local & 1;
         const uint32_t acc_ph = (local >> 1) & 1u;
-        if (!mbar_wait_warp(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc)) { ok = false; break; }
+        if (!mbar_wait_warp(acc_empty_bar(acc), acc_ph ^ 1u, abort_flag, p.status, kTimeoutMmaAcc, wait_limit(p))) { ok = false; break; }
         tcgen05_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * kPairN;
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1u;
-          if (!mbar_wait_warp(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull)) { ok = false; break; }
+          if (!mbar_wait_warp(full_bar(s), ph, abort_flag, p.status, kTimeoutMmaFull, wait_limit(p))) { ok = false; break; }
           tcgen05_fence_after_sync();
           const uint32_t sa = smem_base + s * kStage, sb = sa + kStageA;
           if (elect_one()) {
@@ -229,6 +230,8 @@ pd_status launch_pair_variant(const GemmProblem& g, cudaStream_t s) {
   if (tiles > 0x7fffffff) return PD_ERR_BAD_SHAPE;
   p.num_tiles = (int)tiles;
   p.alpha = g.alpha; p.c_is_f32 = C_F32; p.act = g.act;
+  p.wait_limit_ns = debug_wait_limit_ns();
+  p.withhold_loads = debug_withhold_loads();
 
   auto kernel = gemm_bf16_tcgen05_pair_kernel<B_NK, C_F32>;
   static PerDeviceFlag smem_allowed;  // one per kernel (template instantiation)

@@ -1,9 +1,10 @@
 """A bounded wait that runs out: the kernel must record a code, drain and return, and the library must stay usable.
 
-Every wait inside the tensor-core kernels is bounded.  Here the single-CTA contraction kernel is launched on one
-tile (one CTA, one k-block) with its producer switched off (pd_debug_withhold_loads) and the limit cut to one
-millisecond: the thread that feeds the tensor core waits for an operand stage nobody fills, gives up, and the kernel
-returns.  Nothing faults or hangs: no copy and no product is in flight when the wait gives up."""
+Every wait inside the tensor-core kernels is bounded.  Here the single-CTA contraction kernel (one CTA) and the
+CTA-pair kernel (one pair) are launched on one tile of one k-block with their producers switched off
+(pd_debug_withhold_loads) and the limit cut to one millisecond: the warp that feeds the tensor core waits for an
+operand stage nobody fills, gives up, and the kernel returns.  Nothing faults or hangs: no copy and no product is
+in flight when the wait gives up."""
 import ctypes
 
 import numpy as np
@@ -17,14 +18,15 @@ from parity import dev_bf16, host
 pytestmark = pytest.mark.gpu
 
 
-def test_expired_wait_is_reported_and_the_next_launch_is_correct():
+@pytest.mark.parametrize("tile_mode,M", [(1, 128), (2, 256)], ids=["single_cta_kernel", "cta_pair_kernel"])
+def test_expired_wait_is_reported_and_the_next_launch_is_correct(tile_mode, M):
     from paper_2511_03586_b200 import api
-    M, N, K = 128, 256, 64                                    # one 128 x 256 tile, one k-block
+    N, K = 256, 64                                            # one tile (128 or 256 rows x 256 columns), one k-block
     p = inputs.gemm_integer_inputs(M, N, K, seed=5)
     a, b = dev_bf16(p["a_bits"][0]), dev_bf16(p["b_bits"][0])
     ref = oracle.gemm(p["a"][0], p["b"][0])
     api.pd_clear_device_status()
-    api.pd_set_gemm_tile_mode(1)                               # single-CTA tiles
+    api.pd_set_gemm_tile_mode(tile_mode)
     try:
         api.pd_debug_set_wait_limit_ns(1_000_000)              # 1 ms
         api.pd_debug_withhold_loads(True)
