@@ -41,7 +41,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel at the FFN-up / configured
 # GEMM shape, from the ncu capture summarised in profiles/gemm_bf16_tcgen05_pair_16384x4096x1024.md.  Set to None
 # whenever that kernel changes until the counters are taken again.
-DOMINANT_KERNEL_DRAM_TRAFFIC_BYTES = 42.019840e6 + 78.988800e6
+DOMINANT_KERNEL_DRAM_TRAFFIC_BYTES = 42.002176e6 + 80.332544e6
 METRIC = "achieved HBM GB/s (row ops) and bf16 TFLOP/s (GEMM, layer) as % of roofline"
 
 
