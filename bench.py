@@ -241,7 +241,8 @@ def ops_suite(torch, api, peaks, only: str = ""):
         rowop_entry(f"softmax_{rows}x{cols}", ms, rows * cols * 8, note)
         del xs, ys
 
-    for rows, cols, note in ((4096, 1024, "configured shape"), (16384, 1024, "paper shape"), (4096, 4096, "paper shape")):
+    for rows, cols, note in ((4096, 1024, "configured shape"), (16384, 1024, "paper shape"), (4096, 4096, "paper shape"),
+                             (2048, 24576, "long rows: one 256-thread CTA per row, 24 float4 per thread")):
         if not wanted(f"layernorm_{rows}x{cols}"):
             continue
         p = inputs.layernorm_inputs(rows, cols)

@@ -8,7 +8,9 @@
 // registers (data centred before squaring, mean refined by the mean of the
 // residuals: no E[x^2] - mu^2 cancellation), reduced with warp shuffles.
 //   * cols <= 1024   : one warp per row, two rows per CTA
-//   * cols <= 28672  : one CTA of 64 to 1024 threads per row
+//   * cols <= 16384  : one CTA of 64 to 512 threads per row, 8 float4 per thread
+//   * cols <= 28672  : one CTA of 256 threads per row, 20 to 28 float4 per thread at 128 registers (two rows
+//                      in flight per SM)
 //   * cols <= 262144 : one cluster of 2 to 8 CTAs per row, ceil(cols / 16384) CTAs of 512 threads up to
 //                      131072 columns and ceil(cols / 32768) of 1024 beyond (partial statistics merged
 //                      through distributed shared memory)
@@ -21,8 +23,10 @@
 namespace pd {
 namespace {
 
+constexpr int64_t kFatRowCols = 28672;  // columns one 256-thread CTA holds at 28 float4 per thread
+
 template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA, typename OutT>
-__global__ void __launch_bounds__(THREADS_PER_CTA, THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight
+__global__ void __launch_bounds__(THREADS_PER_CTA, VPT > 8 ? 2 : (THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA)))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight; 128 for the 256-thread CTAs that hold 20 to 28 float4 per thread (rows of 16388 to 28672 columns, two of them in flight per SM)
 layernorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__ gamma,
                             const float* __restrict__ beta, OutT* __restrict__ y, int64_t rows, int cols,
                             float eps) {
@@ -247,11 +251,11 @@ void launch_warp_rows(const float* x, const float* g, const float* b, OutT* y, i
   launch_pdl(kernel, dim3(grid), dim3(kThreads), 0, s, x, g, b, y, rows, cols, eps);
 }
 
-// One CTA of THREADS threads per row, up to 8 float4 per thread.
-template <int THREADS, typename OutT>
+// One CTA of THREADS threads per row, up to VPT float4 per thread.
+template <int THREADS, typename OutT, int VPT = 8>
 void launch_cta_rows(const float* x, const float* g, const float* b, OutT* y, int64_t rows, int cols, float eps,
                      cudaStream_t s) {
-  auto kernel = layernorm_rows_in_registers<8, THREADS, THREADS, OutT>;
+  auto kernel = layernorm_rows_in_registers<VPT, THREADS, THREADS, OutT>;
   const int grid = (int)(rows < 0x7fffffff ? rows : 0x7fffffff);
   launch_pdl(kernel, dim3(grid), dim3(THREADS), 0, s, x, g, b, y, rows, cols, eps);
 }
@@ -264,7 +268,7 @@ pd_status dispatch(const float* x, const float* g, const float* b, OutT* y, int6
   logf("%s %lld x %lld: %s", "layernorm", (long long)rows, (long long)cols,
        !vec_ok ? "scalar three-pass path (unaligned or ragged rows)"
        : cols <= 1024 ? "one warp per row, row in registers"
-       : cols <= 28672 ? "one CTA per row, row in registers"
+       : cols <= kFatRowCols ? "one CTA per row, row in registers"
        : cols <= 262144 ? "one cluster per row, row in registers" : "one CTA per row, streaming passes");
   if (vec_ok && cols <= 1024) {
     const int c = (int)cols;
@@ -272,14 +276,19 @@ pd_status dispatch(const float* x, const float* g, const float* b, OutT* y, int6
     else if (c <= 256) launch_warp_rows<2>(x, g, b, y, rows, c, eps, s);
     else if (c <= 512) launch_warp_rows<4>(x, g, b, y, rows, c, eps, s);
     else launch_warp_rows<8>(x, g, b, y, rows, c, eps, s);
-  } else if (vec_ok && cols <= 28672) {  // beyond (measured): a cluster of 512-thread CTAs, two per SM, is faster
+  } else if (vec_ok && cols <= kFatRowCols) {
     const int c = (int)cols;
     if (c <= 2048) launch_cta_rows<64>(x, g, b, y, rows, c, eps, s);
     else if (c <= 4096) launch_cta_rows<128>(x, g, b, y, rows, c, eps, s);
     else if (c <= 8192) launch_cta_rows<256>(x, g, b, y, rows, c, eps, s);
     else if (c <= 16384) launch_cta_rows<512>(x, g, b, y, rows, c, eps, s);
-    else launch_cta_rows<1024>(x, g, b, y, rows, c, eps, s);
+    // beyond: 256 threads with 20, 24 or 28 float4 each at 128 registers, two rows in flight per SM (one CTA of 1024
+    // threads per SM leaves the memory pipe idle while its row is reduced: 4.0 against 5.8 TB/s at 20480 columns)
+    else if (c <= 20480) launch_cta_rows<256, OutT, 20>(x, g, b, y, rows, c, eps, s);
+    else if (c <= 24576) launch_cta_rows<256, OutT, 24>(x, g, b, y, rows, c, eps, s);
+    else launch_cta_rows<256, OutT, 28>(x, g, b, y, rows, c, eps, s);
   } else if (vec_ok && cols <= 262144 && rows * 8 <= 0x7fffffff) {
+    // (clusters of the 256-thread CTAs above are slower than these: LayerNorm at 65536 columns 3.0 against 4.2 TB/s)
     if (cols <= 131072) {
       const unsigned cl = (unsigned)((cols + 16383) / 16384);
       launch_pdl_cluster(layernorm_rows_cluster<512, OutT>, dim3((unsigned)rows * cl), dim3(512), cl, 0, s, x, g, b, y, rows,

@@ -6,7 +6,7 @@
 // HBM-bound, 8 bytes per element: the row is read once into registers with
 // 128-bit streaming loads, the sum of squares is reduced with warp shuffles (and
 // through shared memory when several warps share a row), and the row is written
-// once.  Same paths as the LayerNorm kernel: a warp (cols <= 1024), a CTA (<= 32768) or a cluster of 2 to 8
+// once.  Same paths as the LayerNorm kernel: a warp (cols <= 1024), a CTA (<= 28672) or a cluster of 2 to 8
 // CTAs (<= 262144) per row, by row length.
 #include "pd_common.cuh"
 
@@ -14,7 +14,7 @@ namespace pd {
 namespace {
 
 template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA>
-__global__ void __launch_bounds__(THREADS_PER_CTA, THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight
+__global__ void __launch_bounds__(THREADS_PER_CTA, VPT > 8 ? 2 : (THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA)))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight; 128 for the 256-thread CTAs that hold 20 to 28 float4 per thread (rows of 16388 to 28672 columns, two of them in flight per SM)
 rmsnorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__ gamma, float* __restrict__ y,
                           int64_t rows, int cols, float eps) {
   constexpr int ROWS_PER_CTA = THREADS_PER_CTA / THREADS_PER_ROW;
@@ -114,11 +114,13 @@ void launch_warp_rows(const float* x, const float* g, float* y, int64_t rows, in
   launch_pdl(rmsnorm_rows_in_registers<VPT, 32, kThreads>, dim3(grid), dim3(kThreads), 0, s, x, g, y, rows, cols, eps);
 }
 
-template <int THREADS>
+template <int THREADS, int VPT = 8>
 void launch_cta_rows(const float* x, const float* g, float* y, int64_t rows, int cols, float eps, cudaStream_t s) {
   const int grid = (int)(rows < 0x7fffffff ? rows : 0x7fffffff);
-  launch_pdl(rmsnorm_rows_in_registers<8, THREADS, THREADS>, dim3(grid), dim3(THREADS), 0, s, x, g, y, rows, cols, eps);
+  launch_pdl(rmsnorm_rows_in_registers<VPT, THREADS, THREADS>, dim3(grid), dim3(THREADS), 0, s, x, g, y, rows, cols, eps);
 }
+
+constexpr int64_t kFatRowCols = 28672;  // columns one 256-thread CTA holds at 28 float4 per thread
 
 }  // namespace
 
@@ -128,19 +130,23 @@ pd_status launch_rmsnorm(const float* x, const float* g, float* y, int64_t rows,
   const int c = (int)cols;
   logf("rmsnorm %lld x %lld: %s", (long long)rows, (long long)cols,
        !vec_ok ? "scalar path (unaligned or ragged rows)" : cols <= 1024 ? "one warp per row, row in registers"
-       : cols <= 32768 ? "one CTA per row, row in registers" : cols <= 262144 ? "one cluster per row, row in registers" : "scalar path");
+       : cols <= 28672 ? "one CTA per row, row in registers" : cols <= 262144 ? "one cluster per row, row in registers" : "scalar path");
   if (vec_ok && cols <= 1024) {
     if (c <= 128) launch_warp_rows<1>(x, g, y, rows, c, eps, s);
     else if (c <= 256) launch_warp_rows<2>(x, g, y, rows, c, eps, s);
     else if (c <= 512) launch_warp_rows<4>(x, g, y, rows, c, eps, s);
     else launch_warp_rows<8>(x, g, y, rows, c, eps, s);
-  } else if (vec_ok && cols <= 32768) {
+  } else if (vec_ok && cols <= kFatRowCols) {
     if (c <= 2048) launch_cta_rows<64>(x, g, y, rows, c, eps, s);
     else if (c <= 4096) launch_cta_rows<128>(x, g, y, rows, c, eps, s);
     else if (c <= 8192) launch_cta_rows<256>(x, g, y, rows, c, eps, s);
     else if (c <= 16384) launch_cta_rows<512>(x, g, y, rows, c, eps, s);
-    else launch_cta_rows<1024>(x, g, y, rows, c, eps, s);
+    // beyond: 256 threads with 20, 24 or 28 float4 each at 128 registers, two rows in flight per SM
+    else if (c <= 20480) launch_cta_rows<256, 20>(x, g, y, rows, c, eps, s);
+    else if (c <= 24576) launch_cta_rows<256, 24>(x, g, y, rows, c, eps, s);
+    else launch_cta_rows<256, 28>(x, g, y, rows, c, eps, s);
   } else if (vec_ok && cols <= 262144 && rows * 8 <= 0x7fffffff) {
+    // (clusters of the 256-thread CTAs above are slower than these: LayerNorm at 65536 columns 3.0 against 4.2 TB/s)
     if (cols <= 131072) {
       const unsigned cl = (unsigned)((cols + 16383) / 16384);
       launch_pdl_cluster(rmsnorm_rows_cluster<512>, dim3((unsigned)rows * cl), dim3(512), cl, 0, s, x, g, y, rows, c, eps);

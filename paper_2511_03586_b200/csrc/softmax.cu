@@ -7,6 +7,8 @@
 // warp shuffles, and written once.
 //   * cols <= 1024            : one warp per row (up to 8 float4 per lane), two rows per CTA
 //   * cols <= 16384           : one CTA of 64 to 512 threads per row (8 float4 per thread)
+//   * cols <= 28672           : one CTA of 256 threads per row, 20 to 28 float4 per thread at 128 registers
+//                               (two rows in flight per SM)
 //   * cols <= 262144          : one cluster of 2 to 8 CTAs per row, ceil(cols / 16384) CTAs of 512 threads up
 //                               to 131072 columns and ceil(cols / 32768) of 1024 beyond (statistics combined
 //                               through distributed shared memory)
@@ -19,11 +21,13 @@ namespace {
 
 #define kNegInf (-INFINITY)
 
+constexpr int64_t kFatRowCols = 28672;  // columns one 256-thread CTA holds at 28 float4 per thread
+
 // One row held by THREADS_PER_ROW threads, VPT float4 each; threads of a row are
 // consecutive lanes.  THREADS_PER_ROW == 32: one warp per row, several rows per
 // CTA.  THREADS_PER_ROW == blockDim.x: one row per CTA.
 template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA, typename OutT>
-__global__ void __launch_bounds__(THREADS_PER_CTA, THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight
+__global__ void __launch_bounds__(THREADS_PER_CTA, VPT > 8 ? 2 : (THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA)))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight; 128 for the 256-thread CTAs that hold 20 to 28 float4 per thread (rows of 16388 to 28672 columns, two of them in flight per SM)
 softmax_rows_in_registers(const float* __restrict__ x, OutT* __restrict__ y, int64_t rows, int cols) {
   constexpr int ROWS_PER_CTA = THREADS_PER_CTA / THREADS_PER_ROW;
   constexpr int NWARPS = THREADS_PER_ROW / 32;
@@ -176,10 +180,10 @@ void launch_warp_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStrea
   launch_pdl(kernel, dim3(grid), dim3(kThreads), 0, s, x, y, rows, cols);
 }
 
-// One CTA of THREADS threads per row, up to 8 float4 per thread.
-template <int THREADS, typename OutT>
+// One CTA of THREADS threads per row, up to VPT float4 per thread.
+template <int THREADS, typename OutT, int VPT = 8>
 void launch_cta_rows(const float* x, OutT* y, int64_t rows, int cols, cudaStream_t s) {
-  auto kernel = softmax_rows_in_registers<8, THREADS, THREADS, OutT>;
+  auto kernel = softmax_rows_in_registers<VPT, THREADS, THREADS, OutT>;
   const int grid = (int)(rows < 0x7fffffff ? rows : 0x7fffffff);
   launch_pdl(kernel, dim3(grid), dim3(THREADS), 0, s, x, y, rows, cols);
 }
@@ -190,7 +194,7 @@ pd_status dispatch(const float* x, OutT* y, int64_t rows, int64_t cols, cudaStre
   logf("%s %lld x %lld: %s", "softmax", (long long)rows, (long long)cols,
        !vec_ok ? "scalar three-pass path (unaligned or ragged rows)"
        : cols <= 1024 ? "one warp per row, row in registers"
-       : cols <= 16384 ? "one CTA per row, row in registers"
+       : cols <= kFatRowCols ? "one CTA per row, row in registers"
        : cols <= 262144 ? "one cluster per row, row in registers" : "one CTA per row, streaming passes");
   if (vec_ok && cols <= 1024) {
     const int c = (int)cols;
@@ -198,13 +202,19 @@ pd_status dispatch(const float* x, OutT* y, int64_t rows, int64_t cols, cudaStre
     else if (c <= 256) launch_warp_rows<2>(x, y, rows, c, s);
     else if (c <= 512) launch_warp_rows<4>(x, y, rows, c, s);
     else launch_warp_rows<8>(x, y, rows, c, s);
-  } else if (vec_ok && cols <= 16384) {  // beyond: two 512-thread CTAs per SM beat one of 1024
+  } else if (vec_ok && cols <= kFatRowCols) {
     const int c = (int)cols;
     if (c <= 2048) launch_cta_rows<64>(x, y, rows, c, s);
     else if (c <= 4096) launch_cta_rows<128>(x, y, rows, c, s);
     else if (c <= 8192) launch_cta_rows<256>(x, y, rows, c, s);
-    else launch_cta_rows<512>(x, y, rows, c, s);
+    else if (c <= 16384) launch_cta_rows<512>(x, y, rows, c, s);
+    // beyond: 256 threads with 20, 24 or 28 float4 each at 128 registers, two rows in flight per SM (one CTA of 1024
+    // threads per SM leaves the memory pipe idle while its row is reduced)
+    else if (c <= 20480) launch_cta_rows<256, OutT, 20>(x, y, rows, c, s);
+    else if (c <= 24576) launch_cta_rows<256, OutT, 24>(x, y, rows, c, s);
+    else launch_cta_rows<256, OutT, 28>(x, y, rows, c, s);
   } else if (vec_ok && cols <= 262144 && rows * 8 <= 0x7fffffff) {
+    // (clusters of the 256-thread CTAs above are slower than these: LayerNorm at 65536 columns 3.0 against 4.2 TB/s)
     if (cols <= 131072) {
       const unsigned cl = (unsigned)((cols + 16383) / 16384);
       launch_pdl_cluster(softmax_rows_cluster<512, OutT>, dim3((unsigned)rows * cl), dim3(512), cl, 0, s, x, y, rows, (int)cols);
