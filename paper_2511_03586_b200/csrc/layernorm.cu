@@ -8,9 +8,9 @@
 // registers (data centred before squaring, mean refined by the mean of the
 // residuals: no E[x^2] - mu^2 cancellation), reduced with warp shuffles.
 //   * cols <= 1024   : one warp per row, two rows per CTA
-//   * cols <= 16384  : one CTA of 64 to 512 threads per row, 8 float4 per thread
-//   * cols <= 28672  : one CTA of 256 threads per row, 20 to 28 float4 per thread at 128 registers (two rows
-//                      in flight per SM)
+//   * cols <= 8192   : one CTA of 64 to 256 threads per row, 8 float4 per thread
+//   * cols <= 28672  : one CTA of 256 threads per row, 12 to 28 float4 per thread at 85 or 128 registers (three
+//                      or two rows in flight per SM)
 //   * cols <= 262144 : one cluster of 2 to 8 CTAs per row, ceil(cols / 16384) CTAs of 512 threads up to
 //                      131072 columns and ceil(cols / 32768) of 1024 beyond (partial statistics merged
 //                      through distributed shared memory)
@@ -26,7 +26,7 @@ namespace {
 constexpr int64_t kFatRowCols = 28672;  // columns one 256-thread CTA holds at 28 float4 per thread
 
 template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA, typename OutT>
-__global__ void __launch_bounds__(THREADS_PER_CTA, VPT > 8 ? 2 : (THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA)))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight; 128 for the 256-thread CTAs that hold 20 to 28 float4 per thread (rows of 16388 to 28672 columns, two of them in flight per SM)
+__global__ void __launch_bounds__(THREADS_PER_CTA, VPT > 12 ? 2 : VPT > 8 ? 3 : (THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA)))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight; 85 / 128 for the 256-thread CTAs that hold 12 / 16 to 28 float4 per thread (rows of 8196 to 28672 columns, three / two of them in flight per SM)
 layernorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__ gamma,
                             const float* __restrict__ beta, OutT* __restrict__ y, int64_t rows, int cols,
                             float eps) {
@@ -281,9 +281,11 @@ pd_status dispatch(const float* x, const float* g, const float* b, OutT* y, int6
     if (c <= 2048) launch_cta_rows<64>(x, g, b, y, rows, c, eps, s);
     else if (c <= 4096) launch_cta_rows<128>(x, g, b, y, rows, c, eps, s);
     else if (c <= 8192) launch_cta_rows<256>(x, g, b, y, rows, c, eps, s);
-    else if (c <= 16384) launch_cta_rows<512>(x, g, b, y, rows, c, eps, s);
-    // beyond: 256 threads with 20, 24 or 28 float4 each at 128 registers, two rows in flight per SM (one CTA of 1024
-    // threads per SM leaves the memory pipe idle while its row is reduced: 4.0 against 5.8 TB/s at 20480 columns)
+    // from 8196 columns on: 256 threads with 12 float4 each (85 registers, three rows in flight per SM) or 16 to 28
+    // (128 registers, two rows in flight); a CTA of 512 or 1024 threads with 8 float4 each leaves the memory pipe idle
+    // while its row is reduced (LayerNorm: 5.7 -> 6.4 TB/s at 12288 columns, 4.0 -> 5.8 at 20480)
+    else if (c <= 12288) launch_cta_rows<256, OutT, 12>(x, g, b, y, rows, c, eps, s);
+    else if (c <= 16384) launch_cta_rows<256, OutT, 16>(x, g, b, y, rows, c, eps, s);
     else if (c <= 20480) launch_cta_rows<256, OutT, 20>(x, g, b, y, rows, c, eps, s);
     else if (c <= 24576) launch_cta_rows<256, OutT, 24>(x, g, b, y, rows, c, eps, s);
     else launch_cta_rows<256, OutT, 28>(x, g, b, y, rows, c, eps, s);

@@ -14,7 +14,7 @@ namespace pd {
 namespace {
 
 template <int VPT, int THREADS_PER_ROW, int THREADS_PER_CTA>
-__global__ void __launch_bounds__(THREADS_PER_CTA, VPT > 8 ? 2 : (THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA)))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight; 128 for the 256-thread CTAs that hold 20 to 28 float4 per thread (rows of 16388 to 28672 columns, two of them in flight per SM)
+__global__ void __launch_bounds__(THREADS_PER_CTA, VPT > 12 ? 2 : VPT > 8 ? 3 : (THREADS_PER_CTA >= 1024 ? 1 : (THREADS_PER_CTA == 128 ? 5 : 1024 / THREADS_PER_CTA)))  // at most 64 registers (1024 threads resident per SM); 96 for the 128-thread CTAs of 4096-column rows, where five CTAs with the compiler free to keep more loads apart measured 3 % faster than eight; 85 / 128 for the 256-thread CTAs that hold 12 / 16 to 28 float4 per thread (rows of 8196 to 28672 columns, three / two of them in flight per SM)
 rmsnorm_rows_in_registers(const float* __restrict__ x, const float* __restrict__ gamma, float* __restrict__ y,
                           int64_t rows, int cols, float eps) {
   constexpr int ROWS_PER_CTA = THREADS_PER_CTA / THREADS_PER_ROW;
@@ -140,8 +140,11 @@ pd_status launch_rmsnorm(const float* x, const float* g, float* y, int64_t rows,
     if (c <= 2048) launch_cta_rows<64>(x, g, y, rows, c, eps, s);
     else if (c <= 4096) launch_cta_rows<128>(x, g, y, rows, c, eps, s);
     else if (c <= 8192) launch_cta_rows<256>(x, g, y, rows, c, eps, s);
-    else if (c <= 16384) launch_cta_rows<512>(x, g, y, rows, c, eps, s);
-    // beyond: 256 threads with 20, 24 or 28 float4 each at 128 registers, two rows in flight per SM
+    // from 8196 columns on: 256 threads with 12 float4 each (85 registers, three rows in flight per SM) or 16 to 28
+    // (128 registers, two rows in flight); a CTA of 512 or 1024 threads with 8 float4 each leaves the memory pipe idle
+    // while its row is reduced (LayerNorm: 5.7 -> 6.4 TB/s at 12288 columns, 4.0 -> 5.8 at 20480)
+    else if (c <= 12288) launch_cta_rows<256, 12>(x, g, y, rows, c, eps, s);
+    else if (c <= 16384) launch_cta_rows<256, 16>(x, g, y, rows, c, eps, s);
     else if (c <= 20480) launch_cta_rows<256, 20>(x, g, y, rows, c, eps, s);
     else if (c <= 24576) launch_cta_rows<256, 24>(x, g, y, rows, c, eps, s);
     else launch_cta_rows<256, 28>(x, g, y, rows, c, eps, s);

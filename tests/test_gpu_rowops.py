@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 TOL = 1e-5
 
 ROWS = (1, 3, 33)
-COLS = (1, 2, 3, 4, 5, 31, 32, 33, 127, 128, 129, 512, 1000, 1024, 1028, 2048, 4096, 5000, 8192, 16384, 16388, 20480, 20484,
+COLS = (1, 2, 3, 4, 5, 31, 32, 33, 127, 128, 129, 512, 1000, 1024, 1028, 2048, 4096, 5000, 8192, 8196, 12288, 12292, 16384, 16388, 20480, 20484,
         24576, 24580, 28672, 28676, 40000, 65536, 100000, 131076, 262144, 262148)
 
 
